@@ -57,14 +57,22 @@ typedef enum {
   TL_ERR_ARCH = 6,      /* the current device is not compute capability 10.x   */
   TL_ERR_CUDA = 7,      /* a CUDA runtime/driver call or a launch failed       */
   TL_ERR_TIMEOUT = 8,   /* a bounded device-side wait gave up (see status word) */
-  TL_ERR_LIMIT = 9      /* tl_e0m4_matmul_noalloc: problem larger than its built-in scratch serves */
+  TL_ERR_LIMIT = 9,     /* tl_e0m4_matmul_noalloc: problem larger than its built-in scratch serves */
+  TL_ERR_KEY = 10       /* tl_e0m4_tuning_set: unknown key                     */
 } tl_status;
 
 typedef enum { TL_F32 = 0, TL_F16 = 1 } tl_dtype;
 
-/* Kernel families the dispatcher of tl_e0m4_matmul chooses between (Section 2.2: one
- * implementation for decoding, one for prefill). */
-typedef enum { TL_KERNEL_DECODE = 0, TL_KERNEL_PREFILL = 1 } tl_kernel;
+/* Section 2.2 has one matmul implementation for the decoding stage (vector-matrix, bound by the
+ * weight bytes) and one for prefill (matrix-matrix, bound by arithmetic).  The stage of a call is
+ * set by M alone: decoding up to 16 tokens, prefill above. */
+typedef enum { TL_STAGE_DECODE = 0, TL_STAGE_PREFILL = 1 } tl_stage;
+
+/* The two kernels tl_e0m4_matmul dispatches to.  TL_KERNEL_REGISTER: the vector-matrix kernel that
+ * builds the weights in registers (mma.sync fragments).  TL_KERNEL_TENSOR: the tcgen05 kernel with
+ * the dequantized weights in tensor memory.  The cut between them lies inside the decoding stage
+ * (measured: the register kernel wins up to 8 tokens). */
+typedef enum { TL_KERNEL_REGISTER = 0, TL_KERNEL_TENSOR = 1 } tl_kernel;
 
 /* Sizes in bytes of the `packed` and `scales` buffers for a [K, N] weight (host only, no
  * CUDA call).  Section 2.3: 4 bits per weight plus a scaling and a bias coefficient per
@@ -130,8 +138,10 @@ tl_status tl_kv_append(void* cache_dev, const void* new_dev, const void* positio
 tl_status tl_e0m4_dequant(const void* packed_dev, const void* scales_dev, int64_t K, int64_t N,
                           int group, void* w_f16_dev, void* stream);
 
-/* Which kernel family tl_e0m4_matmul runs for this shape (host only, no CUDA call):
- * decoding (vector-matrix, bandwidth bound) for M <= 16, prefill (matrix-matrix) above. */
+/* Which of Section 2.2's two stages a call with M tokens belongs to (host only, no CUDA call). */
+tl_stage tl_e0m4_matmul_stage(int64_t M);
+
+/* Which kernel tl_e0m4_matmul really launches for this shape (host only, no CUDA call). */
 tl_kernel tl_e0m4_matmul_kernel(int64_t M, int64_t K, int64_t N);
 
 /* Bytes of device scratch tl_e0m4_matmul needs for this shape (0 = none).  Host only. */
@@ -149,11 +159,14 @@ tl_status tl_e0m4_workspace_init(void* workspace_dev, size_t workspace_bytes, vo
  * workspace_dev / workspace_bytes: scratch of at least tl_e0m4_matmul_workspace(M, K, N)
  * bytes (may be NULL when that is 0), zeroed as tl_e0m4_workspace_init describes; the decode
  * kernels keep split-K partial sums and tile counters there and return it zeroed.
- * The decode kernels use programmatic dependent launch: a call may begin fetching `packed_dev`
- * and `scales_dev` while the previous kernel of the stream is still running if that kernel is
- * a decode kernel of this library, so the weights of a call must not be written by the
- * tl_e0m4_matmul call enqueued immediately before it (x_dev, y_dev and the workspace are
- * ordered as usual). */
+ * The matmul kernels use programmatic dependent launch: a call begins fetching `packed_dev` and
+ * `scales_dev` as soon as the kernels before it on the stream let their successors start, which
+ * every kernel of this library does at its very beginning.  So the weights of a call must be
+ * complete before the kernel that precedes the call on the stream STARTS: weights written by the
+ * kernels enqueued directly before it (a tl_e0m4_quantize, a copy kernel, another matmul) need an
+ * event, a synchronization or any operation that is not a kernel of this library in between.
+ * Weights are static in inference, which is what this rule relies on; x_dev, y_dev, the addend and
+ * the workspace are ordered as usual. */
 tl_status tl_e0m4_matmul(const void* x_dev, const void* packed_dev, const void* scales_dev,
                          void* y_dev, int64_t M, int64_t K, int64_t N, int group,
                          void* workspace_dev, size_t workspace_bytes, void* stream);
@@ -232,7 +245,9 @@ tl_status tl_e0m4_matmul_batch_host(const tl_e0m4_problem* problems_host, int co
  * The call itself allocates and frees nothing.
  * Limits: 1 <= M <= 16 (more tokens than the array has room for per output column are refused
  * with TL_ERR_LIMIT; use tl_e0m4_matmul with a workspace for those); K, N, alignment and `group`
- * as for tl_e0m4_matmul.  Arguments and result are those of tl_e0m4_matmul.
+ * as for tl_e0m4_matmul.  The arguments are those of tl_e0m4_matmul; the result agrees with
+ * tl_e0m4_matmul's within the library's matmul tolerance, not bit for bit (from 9 tokens on the
+ * two entry points run different kernels, and cut panels meet in atomics in either).
  * The first call on each device looks up the array's device address (the device must be
  * current); make that first call outside any stream capture.  Every call clears the array on
  * `stream` before it launches, because the array keeps whatever the previous call left behind.
@@ -307,6 +322,21 @@ tl_status tl_e0m4_device_status(void* stream);
 
 /* Number of kernels this library has launched in this process so far (all entry points). */
 uint64_t tl_e0m4_launch_count(void);
+
+/* Diagnostics and tests (no counterpart in the paper): overrides one launch heuristic for the whole
+ * process until it is set back.  value < 0 restores the library's own choice; key == NULL restores
+ * all of them.  The overrides are read at every call (sizing calls included), never from the
+ * environment.  Keys: "ksplit" (1..8 CTAs share a tile along K in the tensor-core kernel),
+ * "tc_pair" (0 / 1: pairs of CTAs), "tc_big" (0: rounds of 64 k), "tc_mtiles" (1, 2, 4, 8 times the
+ * fewest token tiles), "list_pair" (0 / 1), "batch_tc_min" (first token count of a list that takes
+ * the tensor-core kernel), "register_max_m" (most tokens of a single call on the register kernel,
+ * 1..16), "decode_split" (1 whole panels per CTA, 2 stream-K ranges), "decode_slices" (CTAs per
+ * panel), "decode_ctas_per_sm" (1, 2), "decode_rot_min", "wait_limit_cycles" (SM cycles after
+ * which a device-side wait gives up and raises TL_ERR_TIMEOUT in the status word; about two seconds
+ * by default), "skip_copies" (1: the producers of the matmul kernels issue no copies, so that with
+ * a short wait limit every wait runs out while nothing is in flight: the safe way to see the
+ * time-out path work).  Unknown key: TL_ERR_KEY. */
+tl_status tl_e0m4_tuning_set(const char* key, int64_t value);
 
 /* Static, human-readable name of a status code. */
 const char* tl_status_string(tl_status status);

@@ -16,9 +16,9 @@ Where the paper is silent the readings are (each repeated at its step):
   * the group range is widened to contain 0, so that the bias is a code;
   * the stored scale is the dequantization scale d (w0-units per w1-unit),
     rounded to fp16; the forward scale is its fp32 reciprocal;
-  * "zero the non-intercepted fraction bits of the bias" = truncate the bias
-    to the 4-bit grid;
-  * "ensure that all w1 fall within the range" = clip;
+  * Section 2.3, Quantization: the bias keeps only the fraction bits that
+    become the code, i.e. it is truncated to the 4-bit grid;
+  * the same paragraph wants every w1 inside the binade: w1 is clipped;
   * y1/y2 are sliced from the fp32 bit pattern of w1;
   * w1 = fl32(fl32(w0 * s) + b): two fp32 roundings, no fused multiply-add.
 
@@ -32,7 +32,7 @@ from __future__ import annotations
 
 import numpy as np
 
-GROUP = 128  # group size along K (Section 3.1: "group size of 128")
+GROUP = 128  # group size along K (the default of Section 3.1)
 
 _F32 = np.float32
 

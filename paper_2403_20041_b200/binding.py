@@ -16,13 +16,14 @@ LIB_PATH = os.path.join(_PKG, "libtl_e0m4.so")
 
 TL_OK = 0
 TL_F32, TL_F16 = 0, 1
-TL_KERNEL_DECODE, TL_KERNEL_PREFILL = 0, 1
+TL_KERNEL_REGISTER, TL_KERNEL_TENSOR = 0, 1
+TL_STAGE_DECODE, TL_STAGE_PREFILL = 0, 1
 GROUP = 128
 
 STATUS_NAMES = {
     0: "TL_OK", 1: "TL_ERR_NULL", 2: "TL_ERR_SHAPE", 3: "TL_ERR_ALIGN", 4: "TL_ERR_DTYPE",
     5: "TL_ERR_WORKSPACE", 6: "TL_ERR_ARCH", 7: "TL_ERR_CUDA", 8: "TL_ERR_TIMEOUT",
-    9: "TL_ERR_LIMIT",
+    9: "TL_ERR_LIMIT", 10: "TL_ERR_KEY",
 }
 
 # every symbol include/tl_e0m4.h declares: name -> (restype, argtypes)
@@ -39,6 +40,8 @@ SYMBOLS = {
     "tl_layernorm": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, ctypes.c_float, _vp]),
     "tl_e0m4_dequant": (_int, [_vp, _vp, _i64, _i64, _int, _vp, _vp]),
     "tl_e0m4_matmul_kernel": (_int, [_i64, _i64, _i64]),
+    "tl_e0m4_matmul_stage": (_int, [_i64]),
+    "tl_e0m4_tuning_set": (_int, [ctypes.c_char_p, _i64]),
     "tl_e0m4_matmul_workspace": (_sz, [_i64, _i64, _i64]),
     "tl_e0m4_workspace_init": (_int, [_vp, _sz, _vp]),
     "tl_e0m4_device_status": (_int, [_vp]),
@@ -307,6 +310,16 @@ def tl_layernorm(x, gamma, beta, eps: float, residual=None, sum_out=None, y=None
 
 def tl_e0m4_matmul_kernel(M: int, K: int, N: int) -> int:
     return lib().tl_e0m4_matmul_kernel(M, K, N)
+
+
+def tl_e0m4_matmul_stage(M: int) -> int:
+    return lib().tl_e0m4_matmul_stage(M)
+
+
+def tl_e0m4_tuning_set(key, value: int = -1) -> None:
+    """Overrides one launch heuristic process-wide (diagnostics and tests); value < 0 restores the
+    library's own choice, key None restores all."""
+    _check(lib().tl_e0m4_tuning_set(key.encode() if key is not None else None, int(value)), "tl_e0m4_tuning_set")
 
 
 def tl_e0m4_matmul_workspace(M: int, K: int, N: int) -> int:

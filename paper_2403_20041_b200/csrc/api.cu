@@ -1,13 +1,23 @@
 // extern "C" boundary: argument validation, the M-based dispatcher and the host-buffer variant.
 #include <atomic>
-#include <cstdlib>
+#include <cstring>
 
 #include "common.cuh"
+#include "tuning.h"
 
 namespace tl {
 
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// Overrides set by tl_e0m4_tuning_set; -1 = the library's own choice.
+static std::atomic<int64_t> g_tuning[kTuneCount];
+static struct TuningInit {
+  TuningInit() {
+    for (auto& v : g_tuning) v.store(-1, std::memory_order_relaxed);
+  }
+} g_tuning_init;
+int64_t tune(TuneKey key) { return g_tuning[key].load(std::memory_order_relaxed); }
 
 namespace {
 
@@ -15,6 +25,10 @@ constexpr int64_t kDecodeMaxM = 16;  // Section 2.2: decoding = vector-matrix, p
 // Inside tl_e0m4_matmul two kernels share the range of M: the register-fragment GEMV kernel up to
 // kRegisterMaxM tokens and the tensor-core kernel above.
 constexpr int64_t kRegisterMaxM = 8;
+inline int64_t register_max_m() {
+  const int64_t v = tune(kTuneRegisterMaxM);
+  return v >= 1 && v <= kDecodeMaxM ? v : kRegisterMaxM;
+}
 // Inside tl_e0m4_matmul_batch the GEMV kernel serves up to this many tokens and the tensor-core
 // list kernel the rest (measured on a ChatGLM2-6B-shaped stack: equal at 8 tokens, the tensor-core
 // kernel 1.3x faster at 9 and 1.5x at 16).
@@ -252,12 +266,14 @@ tl_status tl_e0m8_matmul_batch(const tl_e0m4_problem* problems_host, int count, 
 tl_kernel tl_e0m4_matmul_kernel(int64_t M, int64_t K, int64_t N) {
   (void)K;
   (void)N;
-  return M <= kDecodeMaxM ? TL_KERNEL_DECODE : TL_KERNEL_PREFILL;
+  return M <= register_max_m() ? TL_KERNEL_REGISTER : TL_KERNEL_TENSOR;
 }
+
+tl_stage tl_e0m4_matmul_stage(int64_t M) { return M <= kDecodeMaxM ? TL_STAGE_DECODE : TL_STAGE_PREFILL; }
 
 size_t tl_e0m4_matmul_workspace(int64_t M, int64_t K, int64_t N) {
   if (M <= 0 || K <= 0 || N <= 0 || K % kGroup != 0 || N % kTileN != 0) return 0;
-  if (M <= kRegisterMaxM) return decode_workspace_bytes();
+  if (M <= register_max_m()) return decode_workspace_bytes();
   const size_t pre = gemm_tc_workspace_bytes(M, K, N);
   return pre > decode_workspace_bytes() ? pre : decode_workspace_bytes();
 }
@@ -286,9 +302,8 @@ tl_status tl_e0m4_matmul_batch(const tl_e0m4_problem* problems_host, int count, 
   const tl_status st = check_device();
   if (st != TL_OK) return st;
   // Up to kBatchDecodeMaxM tokens the register-fragment kernel streams the list, above it the
-  // tensor-core kernel does (measured crossover; TL_E0M4_BATCH_TC_MIN moves it for tuning).
-  static const char* tc_env = std::getenv("TL_E0M4_BATCH_TC_MIN");
-  const int64_t tc_min = tc_env ? atoi(tc_env) : kBatchDecodeMaxM + 1;
+  // tensor-core kernel does (measured crossover; tl_e0m4_tuning_set("batch_tc_min", m) moves it).
+  const int64_t tc_min = tune(kTuneBatchTcMin) >= 1 ? tune(kTuneBatchTcMin) : kBatchDecodeMaxM + 1;
   const bool tensor = M > kDecodeMaxM || M >= tc_min;
   unsigned int* status = tensor ? device_status_ptr() : nullptr;
   if (tensor && !status) return TL_ERR_CUDA;
@@ -330,7 +345,7 @@ tl_status matmul_any(const void* x_dev, const void* packed_dev, const void* scal
   const cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __half* add = static_cast<const __half*>(addend_dev);
   cudaError_t e;
-  if (M <= kRegisterMaxM) {
+  if (M <= register_max_m()) {
     e = launch_gemv_decode(static_cast<const __half*>(x_dev), static_cast<const uint32_t*>(packed_dev),
                            static_cast<const uint32_t*>(scales_dev), static_cast<__half*>(y_dev), M, K,
                            N, workspace_dev, s, add, swiglu, group, add_stride);
@@ -526,6 +541,23 @@ tl_status tl_e0m4_device_status(void* stream) {
 
 uint64_t tl_e0m4_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+tl_status tl_e0m4_tuning_set(const char* key, int64_t value) {
+  static const char* const names[kTuneCount] = {
+      "ksplit", "tc_pair", "tc_big", "tc_mtiles", "list_pair", "batch_tc_min", "decode_split", "decode_slices",
+      "decode_ctas_per_sm", "decode_rot_min", "wait_limit_cycles", "skip_copies", "register_max_m"};
+  if (!key) {
+    for (auto& v : g_tuning) v.store(-1, std::memory_order_relaxed);
+    return TL_OK;
+  }
+  for (int k = 0; k < kTuneCount; ++k) {
+    if (std::strcmp(key, names[k]) == 0) {
+      g_tuning[k].store(value < 0 ? -1 : value, std::memory_order_relaxed);
+      return TL_OK;
+    }
+  }
+  return TL_ERR_KEY;
+}
+
 const char* tl_status_string(tl_status status) {
   switch (status) {
     case TL_OK: return "ok";
@@ -538,6 +570,7 @@ const char* tl_status_string(tl_status status) {
     case TL_ERR_CUDA: return "CUDA call or kernel launch failed";
     case TL_ERR_TIMEOUT: return "bounded device-side wait expired";
     case TL_ERR_LIMIT: return "problem exceeds the built-in scratch of the no-alloc entry point (M <= 16)";
+    case TL_ERR_KEY: return "unknown tuning key";
   }
   return "unknown status";
 }

@@ -67,8 +67,7 @@ cudaError_t launch_rmsnorm(const __half* x, const __half* r, const __half* gamma
 cudaError_t launch_layernorm(const __half* x, const __half* r, const __half* gamma, const __half* beta, __half* s_out,
                              __half* y, int64_t M, int64_t K, float eps, cudaStream_t stream);
 // Decode kernels.  `workspace` holds decode_workspace_bytes() bytes that are zero on entry and
-// are left zero.  A batch is a list of independent problems sharing M (<= 16); M above 16 in
-// the single-problem launcher is processed in blocks of 16 tokens, one launch each.
+// are left zero.  A batch is a list of independent problems sharing M (<= 16).
 struct DecodeProblem {
   const __half* x;
   const uint32_t* packed;

@@ -44,12 +44,12 @@
 // launch: only weights are touched before griddepcontrol.wait.
 // Every mbarrier wait is bounded; a wait that gives up raises the device status word and the
 // CTA still releases its tensor memory before it exits.
-#include <cstdlib>
 #include <type_traits>
 #include "common.cuh"
 #include "ptx.cuh"
 #include "umma.cuh"
 #include "tc_common.cuh"
+#include "tuning.h"
 
 namespace tl {
 namespace {
@@ -69,6 +69,8 @@ struct TcParams {
   int ksplit;   // CTAs that share one output tile along K (1 = none)
   float* ws;           // split-K scratch: [tile][tok][128 columns] fp32, zero on entry and left zero
   unsigned int* cnt;   // split-K arrival counters: [tile], zero on entry and left zero
+  long long wait_limit;  // SM cycles after which a bounded wait gives up
+  int skip_copies;       // diagnostics: neither producer issues a copy, so every wait runs out
 };
 
 // One unit of work: an output tile (128-column panel x tok tokens) and a slice of the k groups.
@@ -204,14 +206,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
   bool ok = true;
   if (warp == 0) {
     // ------------------------------------------------- producer of packed codes and scale words
-    if (lane == 0) {
+    if (lane == 0 && !p.skip_copies) {
       int ps = 0, pphase = 0, first = 1;
       for (int item = unit; item < total_items && ok; item += units) {
         const TcItem wi = tc_item<SPLIT, PAIR>(p, item, rank);
         const int R = wi.R;
         const size_t tile_base = (size_t)wi.panel * kPanelTiles * ng;
         for (int g = wi.g0; g < wi.g1; ++g) {
-          if (!first && !ptx::mbar_wait_bounded(empty_p + 8 * ps, pphase ^ 1)) { ok = false; break; }
+          if (!first && !ptx::mbar_wait_bounded(empty_p + 8 * ps, pphase ^ 1, p.wait_limit)) { ok = false; break; }
           const size_t tile0 = tile_base + (size_t)g * R;
           const uint32_t pk = pk0 + ps * kSlot;
           if (R > 0) {
@@ -227,7 +229,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
     }
   } else if (warp == 2) {
     // ------------------------------------------------- producer of the token boxes
-    if (lane == 0) {
+    if (lane == 0 && !p.skip_copies) {
       ptx::pdl_wait();
       int s = 0, it = 0;
       for (int item = unit; item < total_items && ok; item += units) {
@@ -236,7 +238,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
         for (int kh = 2 * wi.g0; kh < 2 * wi.g1; kh += HALVES, ++it) {
           // the box was last used by stage it - S
           const int prev = it - S;
-          if (prev >= 0 && !ptx::mbar_wait_bounded(consumed + 8 * (prev & (SA - 1)), (prev / SA) & 1)) {
+          if (prev >= 0 && !ptx::mbar_wait_bounded(consumed + 8 * (prev & (SA - 1)), (prev / SA) & 1, p.wait_limit)) {
             ok = false;
             break;
           }
@@ -266,12 +268,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
     int s = 0, sa = 0, aphase = 0, lt = 0;
     if (PAIR && rank != 0) lt = total_items;  // only CTA 0 of a pair issues
     for (int item = PAIR && rank != 0 ? total_items : unit; item < total_items && ok; item += units, ++lt) {
-      if (lt > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_empty, (lt - 1) & 1))) { ok = false; break; }
+      if (lt > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_empty, (lt - 1) & 1, p.wait_limit))) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const TcItem wi = tc_item<SPLIT, PAIR>(p, item, rank);
       const int stages = (2 / HALVES) * (wi.g1 - wi.g0);
       for (int kh = 0; kh < stages; ++kh) {
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(ready + 8 * sa, aphase))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(ready + 8 * sa, aphase, p.wait_limit))) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t x_st = smem0 + s * x_stage_bytes;
         const uint32_t a_t = t_base + kAccCols + sa * kRoundCols;
@@ -379,8 +381,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
           // slot, four rounds of 128 k ago, has been consumed, the codes of every round up to that
           // one have landed; with at least four packed slots that includes the previous round of
           // the packed slot waited on next.
-          if (sn > 0 && !ptx::mbar_wait_bounded(consumed + 8 * s, (sn - 1) & 1)) { ok = false; break; }
-          if (!ptx::mbar_wait_bounded(full_p + 8 * ps, pphase)) { ok = false; break; }
+          if (sn > 0 && !ptx::mbar_wait_bounded(consumed + 8 * s, (sn - 1) & 1, p.wait_limit)) { ok = false; break; }
+          if (!ptx::mbar_wait_bounded(full_p + 8 * ps, pphase, p.wait_limit)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t pk = pk0 + ps * kSlot;
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kRoundCols;
@@ -425,7 +427,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
       };
       uint4 a_cur[4], a_nxt[4];
       if constexpr (!SPLIT && ADD) load_add(a_cur, 0);
-      if (!ptx::mbar_wait_bounded(acc_full, lt & 1)) { ok = false; break; }
+      if (!ptx::mbar_wait_bounded(acc_full, lt & 1, p.wait_limit)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t t_acc = tmem_base + ((uint32_t)(quad * 32) << 16);
       // Staging tile of this warp: [token 0..31][column 0..31] fp16, so that the global stores are
@@ -668,9 +670,9 @@ TcPlan tc_plan(int64_t M, int64_t K, int64_t N, int bits = 4) {
   const int panels = (nbs + kPanelTiles - 1) / kPanelTiles;
   const int ng = (int)(K / kGroup);
   const double t_item = 3.5;
-  // Tuning aid: TL_E0M4_TC_MTILES=1 / 2 / 4 / 8 fixes the multiple of the fewest token tiles.
-  const char* mt_env = getenv("TL_E0M4_TC_MTILES");
-  const int forced_mult = mt_env ? atoi(mt_env) : 0;
+  // tl_e0m4_tuning_set("tc_mtiles", 1 / 2 / 4 / 8) fixes the multiple of the fewest token tiles.
+  const int64_t mt_set = tune(kTuneTcMtiles);
+  const int forced_mult = (mt_set == 1 || mt_set == 2 || mt_set == 4 || mt_set == 8) ? (int)mt_set : 0;
   int best = 1;
   double best_cost = 1e30;
   pl.tok = 0;
@@ -707,22 +709,20 @@ TcPlan tc_plan(int64_t M, int64_t K, int64_t N, int bits = 4) {
   const bool fewest_tiles = pl.tok == (int)(((M + want - 1) / want + 15) / 16 * 16);  // M was not cut further
   pl.ksplit = best;
   pl.pair = false;
-  // Tuning aid: TL_E0M4_KSPLIT=n forces n slices where the shape allows them.
-  if (const char* e = getenv("TL_E0M4_KSPLIT")) {
-    const int f = atoi(e);
-    if (f >= 1 && f <= 8 && (f == 1 || f * 4 <= ng)) pl.ksplit = f;
+  // tl_e0m4_tuning_set("ksplit", n) forces n slices where the shape allows them.
+  {
+    const int64_t f = tune(kTuneKsplit);
+    if (f >= 1 && f <= 8 && (f == 1 || f * 4 <= ng)) pl.ksplit = (int)f;
   }
   // Pairs: when nothing is split and there is enough work for every SM pair.  The token tile is
   // then a multiple of 32 (the two-CTA MMA's granularity).
-  // Tuning aid: TL_E0M4_TC_PAIR=0 / 1 forces the choice where the shape allows it.
+  // tl_e0m4_tuning_set("tc_pair", 0 / 1) forces the choice where the shape allows it.
   const int pair_tok = (int)(((M + want - 1) / want + 31) / 32 * 32);
   const int pair_tiles = ((panels + 1) / 2) * (int)((M + pair_tok - 1) / pair_tok);
   bool pair = pl.ksplit == 1 && fewest_tiles && panels >= 2 && pair_tok <= kTokTile && M > 128 &&
               pair_tiles >= kPolicySMs / 2;
-  if (const char* e = getenv("TL_E0M4_TC_PAIR")) {
-    if (e[0] == '0') pair = false;
-    if (e[0] == '1') pair = pl.ksplit == 1 && fewest_tiles && panels >= 2 && pair_tok <= kTokTile;
-  }
+  if (tune(kTuneTcPair) == 0) pair = false;
+  if (tune(kTuneTcPair) == 1) pair = pl.ksplit == 1 && fewest_tiles && panels >= 2 && pair_tok <= kTokTile;
   if (pair) {
     pl.pair = true;
     pl.tok = pair_tok;
@@ -730,9 +730,7 @@ TcPlan tc_plan(int64_t M, int64_t K, int64_t N, int bits = 4) {
     pl.tiles = pair_tiles;
   }
   pl.big = !pl.pair && pl.tok <= 128;
-  if (const char* e = getenv("TL_E0M4_TC_BIG")) {  // tuning aid: 0 forces 64-k rounds
-    if (e[0] == '0') pl.big = false;
-  }
+  if (tune(kTuneTcBig) == 0) pl.big = false;  // forces rounds of 64 k
   return pl;
 }
 
@@ -812,6 +810,8 @@ cudaError_t launch_gemm_tc(const __half* x, const uint32_t* packed, const uint32
   p.add = add;
   p.add_stride = add_stride >= 0 ? add_stride : N;
   p.status = status;
+  p.wait_limit = wait_limit_cycles();
+  p.skip_copies = tune(kTuneSkipCopies) == 1;
   p.M = (int)M;
   p.K = (int)K;
   p.N = (int)N;

@@ -21,10 +21,10 @@
 // producer, token producer (one tensor map per problem, two boxes of 64 k per round), four
 // dequantizer groups writing the A operand into tensor memory, one MMA-issuing warp (eight
 // tcgen05.mma per wait and commit), four epilogue warps.  Every mbarrier wait is bounded.
-#include <cstdlib>
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tc_common.cuh"
+#include "tuning.h"
 
 namespace tl {
 namespace {
@@ -58,6 +58,8 @@ struct TcBatchParams {
   int M, tok, count, total_rounds;
   int sx;       // token boxes (of one round) in the ring
   int pslots;   // slots of the packed ring
+  int skip_copies;       // diagnostics: neither producer issues a copy, so every wait runs out
+  long long wait_limit;  // SM cycles after which a bounded wait gives up
 };
 
 // A piece of a CTA's range: groups [g0, g1) of one panel of problem j.
@@ -181,14 +183,14 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
   bool ok = true;
   if (warp == 0) {
     // ------------------------------------------------- producer of packed codes and scale words
-    if (lane == 0) {
+    if (lane == 0 && !p.skip_copies) {
       int ps = 0, pphase = 0, first = 1;
       for (PieceWalk<1> w(p, c0, n_rounds, 0); !w.done() && ok; w.next()) {
         const Piece wi = w.cur();
         const TcBatchProb& q = p.prob[wi.j];
         const size_t tile_base = (size_t)wi.panel * kPanelTiles * wi.ng;
         for (int g = wi.g0; g < wi.g1; ++g) {
-          if (!first && !ptx::mbar_wait_bounded(empty_p + 8 * ps, pphase ^ 1)) { ok = false; break; }
+          if (!first && !ptx::mbar_wait_bounded(empty_p + 8 * ps, pphase ^ 1, p.wait_limit)) { ok = false; break; }
           const size_t tile0 = tile_base + (size_t)g * wi.R;
           const uint32_t pk = pk0 + ps * kSlot;
           ptx::mbar_arrive_expect_tx(full_p + 8 * ps, wi.R * (kTileB + 64 * kSubs));
@@ -200,7 +202,7 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
     }
   } else if (warp == 2) {
     // ------------------------------------------------- producer of the token boxes
-    if (lane == 0) {
+    if (lane == 0 && !p.skip_copies) {
       ptx::pdl_wait();
       int s = 0, sa = 0, it = 0;   // token box and barrier of round it
       int wsa = 0, wphase = 0;     // barrier and phase of round it - S, which used the box last
@@ -209,7 +211,7 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
         const CUtensorMap* map = &p.maps[wi.j];
         for (int g = wi.g0; g < wi.g1; ++g, ++it) {
           if (it >= S) {
-            if (!ptx::mbar_wait_bounded(consumed + 8 * wsa, wphase)) { ok = false; break; }
+            if (!ptx::mbar_wait_bounded(consumed + 8 * wsa, wphase, p.wait_limit)) { ok = false; break; }
             if (++wsa == SA) { wsa = 0; wphase ^= 1; }
           }
           const uint32_t bar = ready + 8 * sa;
@@ -229,12 +231,12 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
     const uint32_t idesc = (1u << 4) | ((uint32_t)(p.tok >> 3) << 17) | ((128u >> 4) << 24);
     int s = 0, sa = 0, aphase = 0, lt = 0;
     for (PieceWalk<1> w(p, c0, n_rounds, 0); !w.done() && ok; w.next(), ++lt) {
-      if (lt > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_empty, (lt - 1) & 1))) { ok = false; break; }
+      if (lt > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_empty, (lt - 1) & 1, p.wait_limit))) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const Piece wi = w.cur();
       const int rounds = wi.g1 - wi.g0;
       for (int r = 0; r < rounds; ++r) {
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(ready + 8 * sa, aphase))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(ready + 8 * sa, aphase, p.wait_limit))) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t x_st = smem0 + s * x_round_bytes;
         const uint32_t a_t = t_base + kBatchAccCols + sa * kRoundCols;
@@ -336,8 +338,8 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
           // groups) from lap to lap: the MMAs retire in order, so it implies that the codes of every
           // round up to six rounds back have landed, and with at least six packed slots no group
           // meets a slot's barrier a whole phase early.
-          if (sn > 0 && !ptx::mbar_wait_bounded(consumed + 8 * s, (sn - 1) & 1)) { ok = false; break; }
-          if (!ptx::mbar_wait_bounded(full_p + 8 * ps, pphase)) { ok = false; break; }
+          if (sn > 0 && !ptx::mbar_wait_bounded(consumed + 8 * s, (sn - 1) & 1, p.wait_limit)) { ok = false; break; }
+          if (!ptx::mbar_wait_bounded(full_p + 8 * ps, pphase, p.wait_limit)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t pk = pk0 + ps * kSlot;
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + kBatchAccCols + s * kRoundCols;
@@ -384,7 +386,7 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
       }
       float* tile_ws = p.ws + (size_t)slot * p.tok * 128;
       __half* y_chunk = q.y + (size_t)wi.panel * 128 + quad * 32 + chunk * 8;
-      if (!ptx::mbar_wait_bounded(acc_full, lt & 1)) { ok = false; break; }
+      if (!ptx::mbar_wait_bounded(acc_full, lt & 1, p.wait_limit)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
       for (int mb = 0; mb < rows_here; mb += 32) {
@@ -568,14 +570,14 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
   bool ok = true;
   if (warp == 0) {
     // ------------------------------------------------- producer of packed codes and scale words
-    if (lane == 0) {
+    if (lane == 0 && !p.skip_copies) {
       int ps = 0, pphase = 0, first = 1;
       for (PieceWalk<kStep> w(p, c0, n_rounds, rank); !w.done() && ok; w.next()) {
         const Piece wi = w.cur();
         const TcBatchProb& q = p.prob[wi.j];
         const size_t tile_base = (size_t)wi.panel * kPanelTiles * wi.ng;
         for (int g = wi.g0; g < wi.g1; ++g) {
-          if (!first && !ptx::mbar_wait_bounded(empty_p + 8 * ps, pphase ^ 1)) { ok = false; break; }
+          if (!first && !ptx::mbar_wait_bounded(empty_p + 8 * ps, pphase ^ 1, p.wait_limit)) { ok = false; break; }
           const size_t tile0 = tile_base + (size_t)g * wi.R;
           const uint32_t pk = pk0 + ps * kSlot;
           if (wi.R > 0) {
@@ -591,7 +593,7 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
     }
   } else if (warp == 2) {
     // ------------------------------------------------- producer of the token boxes
-    if (lane == 0) {
+    if (lane == 0 && !p.skip_copies) {
       ptx::pdl_wait();
       int s = 0, sa = 0, it = 0;   // token box and barrier of round it
       int wsa = 0, wphase = 0;     // barrier and phase of round it - S, which used the box last
@@ -600,7 +602,7 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
         const CUtensorMap* map = &p.maps[wi.j];
         for (int g = wi.g0; g < wi.g1; ++g, ++it) {
           if (it >= S) {
-            if (!ptx::mbar_wait_bounded(consumed + 8 * wsa, wphase)) { ok = false; break; }
+            if (!ptx::mbar_wait_bounded(consumed + 8 * wsa, wphase, p.wait_limit)) { ok = false; break; }
             if (++wsa == SA) { wsa = 0; wphase ^= 1; }
           }
           const uint32_t bar = (ready + 8 * sa) & kLeaderMask;
@@ -628,12 +630,12 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
     int s = 0, sa = 0, aphase = 0, lt = 0;
     // only CTA 0 of a pair issues
     for (PieceWalk<kStep> w(p, c0, PAIR && rank != 0 ? 0 : n_rounds, rank); !w.done() && ok; w.next(), ++lt) {
-      if (lt > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_empty, (lt - 1) & 1))) { ok = false; break; }
+      if (lt > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_empty, (lt - 1) & 1, p.wait_limit))) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const Piece wi = w.cur();
       const int rounds = wi.g1 - wi.g0;
       for (int r = 0; r < rounds; ++r) {
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(ready + 8 * sa, aphase))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(ready + 8 * sa, aphase, p.wait_limit))) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t x_st = smem0 + s * x_round_bytes;
         const uint32_t a_t = t_base + kBatchAccCols + sa * kRoundCols;
@@ -740,8 +742,8 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
           // groups) from lap to lap: the MMAs retire in order, so it implies that the codes of every
           // round up to six rounds back have landed, and with at least six packed slots no group
           // meets a slot's barrier a whole phase early.
-          if (sn > 0 && !ptx::mbar_wait_bounded(consumed + 8 * s, (sn - 1) & 1)) { ok = false; break; }
-          if (!ptx::mbar_wait_bounded(full_p + 8 * ps, pphase)) { ok = false; break; }
+          if (sn > 0 && !ptx::mbar_wait_bounded(consumed + 8 * s, (sn - 1) & 1, p.wait_limit)) { ok = false; break; }
+          if (!ptx::mbar_wait_bounded(full_p + 8 * ps, pphase, p.wait_limit)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t pk = pk0 + ps * kSlot;
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + kBatchAccCols + s * kRoundCols;
@@ -789,7 +791,7 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
       }
       float* tile_ws = p.ws + (size_t)slot * p.tok * 128;
       __half* y_chunk = q.y + (size_t)wi.panel * 128 + quad * 32 + chunk * 8;
-      if (!ptx::mbar_wait_bounded(acc_full, lt & 1)) { ok = false; break; }
+      if (!ptx::mbar_wait_bounded(acc_full, lt & 1, p.wait_limit)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
       for (int mb = 0; mb < rows_here; mb += 32) {
@@ -951,13 +953,14 @@ cudaError_t launch_gemm_tc_batch(const DecodeProblem* probs, int count, int M, v
   if (sms <= 0 || sms > kBatchPolicySMs) sms = kBatchPolicySMs;
   // Pairs of CTAs from 81 tokens on: measured on ChatGLM2-6B- and Gemma-2B-shaped lists they are
   // 3-7 % faster from 96 tokens, equal at 72-80 and 8 % slower at 32 (the cluster-wide hand-overs
-  // cost what the halved MMA count saves).  Tuning aid: TL_E0M4_LIST_PAIR=0 / 1 forces the choice.
-  const char* pair_env = getenv("TL_E0M4_LIST_PAIR");
-  const bool pair = pair_env ? pair_env[0] == '1' : M > 80;
+  // cost what the halved MMA count saves).  tl_e0m4_tuning_set("list_pair", 0 / 1) forces the choice.
+  const bool pair = tune(kTuneListPair) >= 0 ? tune(kTuneListPair) == 1 : M > 80;
   for (int j0 = 0; j0 < count; j0 += kMaxTcBatch) {
     const int n = count - j0 < kMaxTcBatch ? count - j0 : kMaxTcBatch;
     TcBatchParams p;
     p.status = status;
+    p.wait_limit = wait_limit_cycles();
+    p.skip_copies = tune(kTuneSkipCopies) == 1;
     p.M = M;
     p.tok = pair ? (M + 31) / 32 * 32 : (M + 15) / 16 * 16;  // the two-CTA MMA takes tokens in steps of 32
     p.count = n;

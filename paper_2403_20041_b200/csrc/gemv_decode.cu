@@ -27,10 +27,11 @@
 //   * Programmatic dependent launch: the kernel lets its successor start at once, and itself
 //     prefetches weights (which no predecessor writes) before it waits for its predecessor;
 //     activations, outputs and scratch are touched only after that wait.
-#include <cstdlib>
+#include <atomic>
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "tuning.h"
 
 namespace tl {
 namespace {
@@ -82,6 +83,8 @@ struct DecodeParams {
   const __half* add;      // single-problem launches only: optional fp16 [M, N] added to the product
                           // before the one rounding (may be y); NULL otherwise
   long long add_stride;   // elements between the addend's token rows: N, or 0 for a bias row shared by all tokens
+  long long wait_limit;   // SM cycles after which a bounded wait gives up
+  int skip_copies;        // diagnostics: the producer issues nothing, so every wait runs out
 };
 
 // silu(g) * u in fp32 (Section 2.2's element-wise fusion for gated MLPs)
@@ -231,7 +234,7 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------------- producer
-    if (lane != 0) return;
+    if (lane != 0 || p.skip_copies) return;
     const uint32_t ring_s = ptx::smem_u32(ring);
     auto issue_w = [&](const StageWalk<NB>& w, int s) {
       const Prob& q = p.prob[w.j];
@@ -271,7 +274,7 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
     // steady state: refill a stage as soon as the consumers have released it
     int s = 0, phase = 0;
     while (!w.done()) {
-      if (!ptx::mbar_wait_bounded(empty0 + 8 * s, phase)) {
+      if (!ptx::mbar_wait_bounded(empty0 + 8 * s, phase, p.wait_limit)) {
         atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
         return;
       }
@@ -294,7 +297,7 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
     const int sub = lane >> 3, part = lane & 7;  // group of the stage, 16-halves slice of its 128 k
     const uint32_t ring_h = ptx::smem_u32(ring);
     for (StageWalk<NB> w(p, c0, n_chunks); !w.done(); w.next()) {
-      if (!ptx::mbar_wait_bounded(xbar0 + 8 * s, phase)) {
+      if (!ptx::mbar_wait_bounded(xbar0 + 8 * s, phase, p.wait_limit)) {
         if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
         return;
       }
@@ -380,7 +383,7 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
     const int rest = q.nbs - kPanelTiles * w.panel;
     const int R = rest < kPanelTiles ? rest : kPanelTiles;
     const int groups = w.groups();
-    if (!ptx::mbar_wait_bounded(full0 + 8 * s, phase)) {
+    if (!ptx::mbar_wait_bounded(full0 + 8 * s, phase, p.wait_limit)) {
       if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
       return;  // every wait in this kernel is bounded, so the other warps leave as well
     }
@@ -665,7 +668,8 @@ cudaError_t launch_one(const DecodeParams<NB>& p, int grid, size_t smem, cudaStr
 template <int NB, int G = kGroup>
 cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* workspace,
                          cudaStream_t stream) {
-  static const char* split_env = std::getenv("TL_E0M4_DECODE_SPLIT");  // "panel" | "stream" | "c<s>" (tuning aid)
+  const int64_t split_mode = tune(kTuneDecodeSplit);   // 1 = whole panels, 2 = stream-K ranges (tl_e0m4_tuning_set)
+  const int64_t forced_slices = tune(kTuneDecodeSlices);
   const int sms = sm_count();
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
@@ -676,6 +680,8 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
   p.count = count;
   p.add = count == 1 ? probs[0].add : nullptr;
   p.add_stride = count == 1 && probs[0].add_stride >= 0 ? probs[0].add_stride : probs[0].N;
+  p.wait_limit = wait_limit_cycles();
+  p.skip_copies = tune(kTuneSkipCopies) == 1;
   long long total = 0;
   for (int j = 0; j < count; ++j) {
     Prob& q = p.prob[j];
@@ -695,8 +701,7 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
   p.total_chunks = (int)total;
 
   // grid: one CTA per SM, fewer when there is less than one chunk per SM
-  static const char* cta_env = std::getenv("TL_E0M4_DECODE_CTAS_PER_SM");  // tuning aid
-  const int per_sm = cta_env ? atoi(cta_env) : 2;
+  const int per_sm = tune(kTuneDecodeCtasPerSm) == 1 ? 1 : 2;
   int grid = p.total_chunks < per_sm * sms ? p.total_chunks : per_sm * sms;
   if (grid > kMaxSlots - 1) grid = kMaxSlots - 1;
   p.unit = 1;
@@ -705,11 +710,11 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
     const int panels = p.prob[0].panels;
     const int per = (panels + grid - 1) / grid;
     bool aligned = panels >= grid && (double)panels / ((double)per * grid) >= 0.97;
-    if (split_env && split_env[0] == 'p') {
+    if (split_mode == 1) {
       aligned = true;
       if (panels < grid) grid = panels;
     }
-    if (split_env && split_env[0] == 's') aligned = false;
+    if (split_mode == 2) aligned = false;
     if (aligned) p.unit = p.prob[0].ng;
     // With fewer panels than CTAs every panel gets its own s CTAs, each taking one slice of the
     // panel's groups: a CTA then flushes one partial tile instead of the two of a range that
@@ -718,11 +723,11 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
     // (up to 1.4x faster than the stream-K ranges), except that two slices of at most 8 groups
     // lose to whole panels.
     int slices = 0;
-    if (panels < grid && !split_env) {
+    if (panels < grid && split_mode < 0 && forced_slices < 0) {
       slices = grid / panels < p.prob[0].ng ? grid / panels : p.prob[0].ng;
       if (slices == 2 && p.prob[0].ng <= 16) slices = 1;
     }
-    if (split_env && split_env[0] == 'c') slices = atoi(split_env + 1);  // "c<s>": s CTAs per panel
+    if (forced_slices > 0 && split_mode < 0) slices = (int)forced_slices;
     if (slices > 0 && slices <= p.prob[0].ng && (long long)panels * slices <= grid) {
       p.unit = -slices;
       grid = panels * slices;
@@ -736,8 +741,8 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
   stages = stages > kMaxStages ? kMaxStages : (stages < 2 ? 2 : stages);
   p.stages = stages;
   const size_t smem = 128 + (size_t)stages * p.stage_bytes + 3 * kMaxStages * sizeof(uint64_t) + 16 + 64;
-  static const char* rot_env = std::getenv("TL_E0M4_DECODE_ROT_MIN");  // tuning aid
-  const int rot_min = rot_env ? atoi(rot_env) : 5;  // measured crossover: the selects cost more than the conflicts below
+  // measured crossover: below five tokens the selects cost more than the conflicts they avoid
+  const int rot_min = tune(kTuneDecodeRotMin) >= 0 ? (int)tune(kTuneDecodeRotMin) : 5;
   cudaError_t e;
   if constexpr (NB == 1) {
     if (p.add) {
@@ -820,16 +825,17 @@ cudaError_t launch_gemv_decode_builtin(const __half* x, const uint32_t* packed, 
                                        __half* y, int M, int64_t K, int64_t N, cudaStream_t stream, int group) {
   // In host code `g_builtin_scratch` is only a handle; the kernel needs the device address,
   // which is looked up once per device while that device is current.
-  static void* address[64] = {nullptr};
+  // (Host threads may race to fill an entry; they all store the same address, atomically.)
+  static std::atomic<void*> address[64];
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  void* ptr = (dev >= 0 && dev < 64) ? address[dev] : nullptr;
+  void* ptr = (dev >= 0 && dev < 64) ? address[dev].load(std::memory_order_acquire) : nullptr;
   if (!ptr) {
     e = cudaGetSymbolAddress(&ptr, g_builtin_scratch);
     if (e != cudaSuccess) return e;
     if (!ptr) return cudaErrorUnknown;
-    if (dev >= 0 && dev < 64) address[dev] = ptr;
+    if (dev >= 0 && dev < 64) address[dev].store(ptr, std::memory_order_release);
   }
   // The array keeps whatever the previous call left (zero after a call that ran to completion,
   // anything after one that was cut short), so it is cleared on the stream before every launch.

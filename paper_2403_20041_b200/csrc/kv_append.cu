@@ -21,19 +21,20 @@ kv_append_kernel(uint4* __restrict__ cache, const uint4* __restrict__ fresh, con
   // positions) may be the previous kernel's output, so they are read after griddepcontrol.wait.
   ptx::pdl_launch_dependents();
   ptx::pdl_wait();
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
   const long long per_b = (long long)H * S * vec_per_row;
-  const int b = (int)(i / per_b);
-  const long long r = i - (long long)b * per_b;
-  const int h = (int)(r / ((long long)S * vec_per_row));
-  const long long in_head = r - (long long)h * S * vec_per_row;  // vector inside the S new rows of (b, h)
-  const int p = pos[b];
-  if (p < 0 || p + S > L) {
-    if (in_head == 0 && h == 0) atomicExch(status, (unsigned)TL_ERR_SHAPE);
-    return;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int b = (int)(i / per_b);
+    const long long r = i - (long long)b * per_b;
+    const int h = (int)(r / ((long long)S * vec_per_row));
+    const long long in_head = r - (long long)h * S * vec_per_row;  // vector inside the S new rows of (b, h)
+    const int p = pos[b];
+    // S <= L is checked on the host, so L - S cannot wrap whatever the position holds
+    if (p < 0 || p > L - S) {
+      if (in_head == 0 && h == 0) atomicExch(status, (unsigned)TL_ERR_SHAPE);
+      continue;
+    }
+    cache[(((long long)b * H + h) * L + p) * vec_per_row + in_head] = fresh[i];
   }
-  cache[(((long long)b * H + h) * L + p) * vec_per_row + in_head] = fresh[i];
 }
 
 }  // namespace
@@ -42,7 +43,9 @@ cudaError_t launch_kv_append(void* cache, const void* fresh, const int* pos, int
                              int64_t D, unsigned int* status, cudaStream_t stream) {
   const int vec_per_row = (int)(D / 8);
   const long long total = (long long)B * H * S * vec_per_row;
-  const unsigned grid = (unsigned)((total + 255) / 256);
+  // one vector per thread up to 2^22 blocks, a grid-stride loop beyond (the grid's x limit is 2^31 - 1)
+  const long long blocks = (total + 255) / 256;
+  const unsigned grid = (unsigned)(blocks < (1LL << 22) ? blocks : (1LL << 22));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(256);

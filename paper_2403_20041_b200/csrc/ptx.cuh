@@ -45,15 +45,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after about `kWaitLimitCycles` SM cycles and reports false, so that a
-// lost signal can never hang the GPU.  Callers set an error flag and leave.
-constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 2 GHz
-
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+// Bounded wait: gives up after about `limit_cycles` SM cycles and reports false, so that a lost
+// signal can never hang the GPU.  Callers set an error flag and leave.  The limit is a launch
+// parameter of every kernel (about two seconds by default).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit_cycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitLimitCycles) return false;
+    if (clock64() - t0 > limit_cycles) return false;
   }
   return true;
 }

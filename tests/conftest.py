@@ -34,3 +34,10 @@ def lib():
     from paper_2403_20041_b200 import binding
 
     return binding
+
+
+@pytest.fixture
+def tuning(lib):
+    """Sets launch-heuristic overrides through tl_e0m4_tuning_set and restores all of them afterwards."""
+    yield lib.tl_e0m4_tuning_set
+    lib.tl_e0m4_tuning_set(None)

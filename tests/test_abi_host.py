@@ -37,11 +37,33 @@ def test_packed_sizes(lib):
         assert err.value.status == 2  # TL_ERR_SHAPE
 
 
-def test_dispatcher_switches_at_sixteen_tokens(lib):
-    for M in (1, 2, 8, 16):
-        assert lib.tl_e0m4_matmul_kernel(M, 4096, 4096) == lib.TL_KERNEL_DECODE
+def test_stage_switches_at_sixteen_tokens_and_kernel_at_eight(lib):
+    for M in (1, 2, 8, 9, 16):
+        assert lib.tl_e0m4_matmul_stage(M) == lib.TL_STAGE_DECODE
     for M in (17, 64, 128, 4096):
-        assert lib.tl_e0m4_matmul_kernel(M, 4096, 4096) == lib.TL_KERNEL_PREFILL
+        assert lib.tl_e0m4_matmul_stage(M) == lib.TL_STAGE_PREFILL
+    # what really runs: the register kernel up to 8 tokens, the tensor-core kernel from 9
+    for M in (1, 2, 8):
+        assert lib.tl_e0m4_matmul_kernel(M, 4096, 4096) == lib.TL_KERNEL_REGISTER
+    for M in (9, 16, 17, 4096):
+        assert lib.tl_e0m4_matmul_kernel(M, 4096, 4096) == lib.TL_KERNEL_TENSOR
+
+
+def test_tuning_overrides_are_read_by_sizing_and_dispatch_and_can_be_restored(lib):
+    L = lib.lib()
+    assert L.tl_e0m4_tuning_set(b"no_such_key", 1) == 10  # TL_ERR_KEY
+    try:
+        lib.tl_e0m4_tuning_set("register_max_m", 16)
+        assert lib.tl_e0m4_matmul_kernel(12, 4096, 4096) == lib.TL_KERNEL_REGISTER
+        lib.tl_e0m4_tuning_set("register_max_m", -1)
+        assert lib.tl_e0m4_matmul_kernel(12, 4096, 4096) == lib.TL_KERNEL_TENSOR
+        base = lib.tl_e0m4_matmul_workspace(200, 2048, 512)
+        lib.tl_e0m4_tuning_set("ksplit", 4)
+        forced = lib.tl_e0m4_matmul_workspace(200, 2048, 512)
+        assert forced > 0 and forced >= base
+    finally:
+        lib.tl_e0m4_tuning_set(None)
+    assert lib.tl_e0m4_matmul_workspace(200, 2048, 512) == base
 
 
 def test_argument_errors_come_back_before_any_launch(lib):

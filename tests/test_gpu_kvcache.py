@@ -57,3 +57,18 @@ def test_rows_beyond_the_cache_are_refused_without_a_fault(lib, dev):
     with pytest.raises(lib.TlError):                     # more new rows than the cache has: refused on the host
         lib.tl_kv_append(c, torch.zeros((B, H, L + 1, D), dtype=torch.float16, device=dev),
                          torch.zeros(B, dtype=torch.int32, device=dev))
+
+
+@pytest.mark.parametrize("bad", [2**31 - 1, 2**31 - 2, -(2**31), -1, 6])
+def test_positions_at_the_ends_of_int32_are_refused(lib, dev, bad):
+    # position + S would wrap around in 32-bit arithmetic; the guard compares position with L - S
+    # instead, skips the entry's stores and raises the status word
+    B, H, L, S, D = 2, 2, 8, 3, 16
+    c = torch.ones((B, H, L, D), dtype=torch.float16, device=dev)
+    new = torch.full((B, H, S, D), 2.0, dtype=torch.float16, device=dev)
+    lib.tl_kv_append(c, new, torch.tensor([bad, 5], dtype=torch.int32, device=dev))
+    torch.cuda.synchronize()
+    out = c.cpu().numpy()
+    assert (out[0] == 1.0).all()
+    assert (out[1, :, 5:8] == 2.0).all() and (out[1, :, :5] == 1.0).all()
+    assert lib.tl_e0m4_device_status() == 2

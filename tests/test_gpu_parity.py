@@ -271,18 +271,18 @@ def test_tensor_core_split_k_leaves_workspace_zero(lib, dev, M, K, N):
 
 @pytest.mark.parametrize("ks", [2, 3, 4])
 @pytest.mark.parametrize("M,K,N", [(9, 2048, 272), (200, 2048, 512), (300, 2176, 144), (520, 2560, 400)])
-def test_tensor_core_split_k_forced(lib, dev, monkeypatch, ks, M, K, N):
+def test_tensor_core_split_k_forced(lib, dev, tuning, ks, M, K, N):
     # the tuning override forces the number of k slices (read at every call), so that ragged
     # panels, several token tiles and uneven group slices all go through the shared-tile path
-    monkeypatch.setenv("TL_E0M4_KSPLIT", str(ks))
+    tuning("ksplit", ks)
     _split_case(lib, dev, M, K, N, seed=workloads.seed_for("ks", ks, M, K, N))
 
 
 @pytest.mark.parametrize("M", [255, 256, 257, 300, 513, 1030])
-def test_tensor_core_token_tile_boundaries(lib, dev, monkeypatch, M):
+def test_tensor_core_token_tile_boundaries(lib, dev, tuning, M):
     # M around the 256-token tile: equal tiles of a multiple of 16 tokens with a ragged last
     # one, 17 column blocks (two full panels and one of a single block), an odd number of groups
-    monkeypatch.setenv("TL_E0M4_KSPLIT", "1")
+    tuning("ksplit", 1)
     y, y_ref = _matmul_case(lib, dev, M, 640 + 128, 272, seed=workloads.seed_for("tb", M), outliers=0.01)
     assert y.shape == (M, 272)
     assert_matmul_close(y, y_ref)
@@ -423,8 +423,8 @@ def test_matmul_add_matches_oracle(lib, dev, M, K, N):
 
 
 @pytest.mark.parametrize("ks", [2, 4])
-def test_matmul_add_with_split_k(lib, dev, monkeypatch, ks):
-    monkeypatch.setenv("TL_E0M4_KSPLIT", str(ks))
+def test_matmul_add_with_split_k(lib, dev, tuning, ks):
+    tuning("ksplit", ks)
     M, K, N = 200, 2048, 400
     w_np = workloads.weights(K, N, seed=61)
     x_np = workloads.activations(M, K, seed=62, outlier_fraction=0.01)
@@ -485,8 +485,8 @@ def test_matmul_swiglu_matches_oracle(lib, dev, M, K, F):
 
 
 @pytest.mark.parametrize("ks", [2, 4])
-def test_matmul_swiglu_with_split_k(lib, dev, monkeypatch, ks):
-    monkeypatch.setenv("TL_E0M4_KSPLIT", str(ks))
+def test_matmul_swiglu_with_split_k(lib, dev, tuning, ks):
+    tuning("ksplit", ks)
     M, K, F = 200, 2048, 200
     x, packed, scales, y_ref = _swiglu_case(lib, dev, M, K, F, seed=81)
     ws = lib.tl_e0m4_workspace(lib.tl_e0m4_matmul_workspace(M, K, 2 * F), dev)
@@ -496,9 +496,9 @@ def test_matmul_swiglu_with_split_k(lib, dev, monkeypatch, ks):
     assert_matmul_close(_to_np(y), y_ref)
 
 
-def test_matmul_swiglu_paired_ctas(lib, dev, monkeypatch):
-    monkeypatch.setenv("TL_E0M4_TC_PAIR", "1")
-    monkeypatch.setenv("TL_E0M4_KSPLIT", "1")
+def test_matmul_swiglu_paired_ctas(lib, dev, tuning):
+    tuning("tc_pair", 1)
+    tuning("ksplit", 1)
     x, packed, scales, y_ref = _swiglu_case(lib, dev, 300, 1024, 200, seed=85)   # 400 columns: 4 panels, the last of one block
     y = lib.tl_e0m4_matmul_swiglu(x, packed, scales, 400)
     torch.cuda.synchronize()
@@ -506,7 +506,7 @@ def test_matmul_swiglu_paired_ctas(lib, dev, monkeypatch):
 
 
 # ---------------------------------------------------------------- seeded sweep over shapes, modes and epilogues
-def test_seeded_sweep_of_shapes_modes_and_epilogues(lib, dev, monkeypatch):
+def test_seeded_sweep_of_shapes_modes_and_epilogues(lib, dev, tuning):
     """Fifty seeded cases: M across both kernels and the tile boundaries, K of 1..24 groups, N of
     1..70 column blocks, split-K forced or not, paired CTAs forced or not, each of the three
     epilogues; every result against the oracle."""
@@ -516,16 +516,16 @@ def test_seeded_sweep_of_shapes_modes_and_epilogues(lib, dev, monkeypatch):
     for it in range(50):
         M = rnd.choice([1, 2, 5, 8, 9, 15, 16, 17, 31, 33, 64, 100, 127, 128, 129, 200, 255, 256, 257, 300, 513, 700])
         K, N = 128 * rnd.randint(1, 24), 16 * rnd.randint(1, 70)
-        monkeypatch.delenv("TL_E0M4_KSPLIT", raising=False)
-        monkeypatch.delenv("TL_E0M4_TC_PAIR", raising=False)
+        tuning("ksplit", -1)
+        tuning("tc_pair", -1)
         mode = rnd.choice(["auto", "ks", "pair", "nopair"])
         if mode == "ks":
-            monkeypatch.setenv("TL_E0M4_KSPLIT", str(rnd.choice([1, 2, 3, 4, 6, 8])))
+            tuning("ksplit", rnd.choice([1, 2, 3, 4, 6, 8]))
         elif mode == "pair":
-            monkeypatch.setenv("TL_E0M4_TC_PAIR", "1")
-            monkeypatch.setenv("TL_E0M4_KSPLIT", "1")
+            tuning("tc_pair", 1)
+            tuning("ksplit", 1)
         elif mode == "nopair":
-            monkeypatch.setenv("TL_E0M4_TC_PAIR", "0")
+            tuning("tc_pair", 0)
         epi = rnd.choice(["plain", "plain", "add", "swiglu"])
         w_np = workloads.weights(K, N, seed=1000 + it)
         x_np = workloads.activations(M, K, seed=2000 + it, outlier_fraction=0.01)
@@ -622,8 +622,8 @@ def test_matmul_bias_matches_oracle(lib, dev, M, K, N):
 
 
 @pytest.mark.parametrize("ks", [2, 4])
-def test_matmul_bias_with_split_k(lib, dev, monkeypatch, ks):
-    monkeypatch.setenv("TL_E0M4_KSPLIT", str(ks))
+def test_matmul_bias_with_split_k(lib, dev, tuning, ks):
+    tuning("ksplit", ks)
     M, K, N = 200, 2048, 512
     w_np = workloads.weights(K, N, seed=31)
     x_np = workloads.activations(M, K, seed=32)
@@ -636,9 +636,9 @@ def test_matmul_bias_with_split_k(lib, dev, monkeypatch, ks):
 
 @pytest.mark.parametrize("pair", ["0", "1"])
 @pytest.mark.parametrize("M", [9, 33, 70, 97, 128])
-def test_list_kernel_with_and_without_paired_ctas(lib, dev, monkeypatch, pair, M):
+def test_list_kernel_with_and_without_paired_ctas(lib, dev, tuning, pair, M):
     # both forms of the tensor-core list kernel at every token count, odd panel counts included
-    monkeypatch.setenv("TL_E0M4_LIST_PAIR", pair)
+    tuning("list_pair", int(pair))
     shapes = [(1408, 272), (256, 400), (2048, 256), (384, 48), (2048, 2048), (640, 128), (13696, 144)]
     ws = lib.tl_e0m4_workspace(lib.tl_e0m4_matmul_batch_workspace(), dev)
     probs, refs = [], []

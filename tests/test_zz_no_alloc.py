@@ -4,16 +4,19 @@ Some users of this library cannot call cudaMalloc when they need a matmul: an in
 that gave its whole device pool to a framework allocator at start-up, a latency-critical loop
 that must not trigger cudaMalloc's device synchronization, a plug-in whose host forbids
 allocation.  For them `tl_e0m4_matmul_noalloc` keeps the decode kernel's scratch in an array
-inside the library.  This test calls it through the C ABI, twice in a row on the same stream,
+inside the library.  The first test calls it through the C ABI, twice in a row on the same stream,
 and checks each result against `tl_e0m4_matmul` (which takes its scratch from the caller) within
 the tolerance the parity tests use; the shape is one whose column panels are split between
 CTAs, so the scratch is really exercised, and the second call finds the array as the first
-left it.
+left it.  The second test covers the entry point's whole range of token counts (1 to 16: above
+8 tokens it is the only default route into the register kernel's two-block form), every group
+size and a last panel of fewer than eight column blocks, against the CPU oracle.
 """
 
 import numpy as np
 import pytest
 
+import oracle
 from paper_2403_20041_b200 import workloads
 
 torch = pytest.importorskip("torch")
@@ -55,6 +58,31 @@ def test_noalloc_entry_point_matches_workspace_entry_point(lib):
     torch.cuda.synchronize()
     _close(y1.cpu().numpy(), ref1.cpu().numpy())
     _close(y2.cpu().numpy(), ref2.cpu().numpy())
+    assert lib.tl_e0m4_device_status() == 0
+
+
+@pytest.mark.parametrize("group", [128, 64, 32])
+@pytest.mark.parametrize("M", [1, 8, 9, 12, 16])
+def test_noalloc_entry_point_matches_oracle_over_its_whole_range(lib, M, group):
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    dev = torch.device("cuda:0")
+    # 2128 = 16 full panels + one of five column blocks; 17 panels over ~300 CTAs: every panel is cut
+    # between CTAs and meets in the built-in scratch
+    K, N = 2048, 2128
+    w_np = workloads.weights(K, N, workloads.seed_for("noalloc", group))
+    codes, d_h, b_h = oracle.quantize(w_np, group=group)
+    w_hat = oracle.dequantize(codes, d_h, b_h, group=group)
+    packed, scales = lib.tl_e0m4_quantize(torch.from_numpy(w_np).to(dev), group=group)
+    xs = [workloads.activations(M, K, workloads.seed_for("noalloc", "x", M, i)) for i in range(2)]
+    xd = [torch.from_numpy(x).to(dev) for x in xs]
+    ys = [torch.full((M, N), float("nan"), dtype=torch.float16, device=dev) for _ in range(2)]
+    torch.cuda.synchronize()
+    for x, y in zip(xd, ys):  # two calls in a row on one stream
+        lib.tl_e0m4_matmul_noalloc(x, packed, scales, y, group=group)
+    torch.cuda.synchronize()
+    for x, y in zip(xs, ys):
+        _close(y.cpu().numpy(), oracle.matmul(x, w_hat))
     assert lib.tl_e0m4_device_status() == 0
 
 
