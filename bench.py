@@ -1,21 +1,25 @@
 #!/usr/bin/env python
 """Benchmark of the E0M4 weight-only FP4 matmul on B200.
 
-One "step" is one decode token's worth of matmuls: every matrix of every layer of a
-Gemma-2B-shaped stack (18 layers x 7 matrices, M = 1, each with its own activations) multiplied
-once.  The headline runs the step as one tl_e0m4_matmul_batch call (the matrices of the synthetic
-stack are independent problems); `per_call` gives the same step as one tl_e0m4_matmul call per
-matrix.  Both are replayed as CUDA graphs.  The packed weights of the stack (about 1.05 GB) are
-far larger than L2, so every step streams them from HBM.
+One "step" is one decode token's worth of matmuls: every matrix of every layer of the 14B-class
+stack (40 layers x 4 matrices, M = 1, each with its own activations; 6.7 GB of packed weights, the
+largest configuration) multiplied once.  The headline runs the step as one tl_e0m4_matmul_batch
+call (the matrices of the synthetic stack are independent problems; one persistent kernel per 192
+problems); `per_call` gives the same step as one tl_e0m4_matmul call per matrix.  Both are replayed
+as CUDA graphs.  The packed weights are far larger than L2, so every step streams them from HBM.
 
 Prints ONE JSON line (rank 0).  `value` is algorithmic GB/s over all GPUs:
-(packed codes + scales + x + y bytes of a step) / step time.  Extra keys: `roofline`
-(decode kernel against the measured HBM copy bandwidth), `prefill` (TFLOP/s of the
-matrix-matrix path on a ChatGLM2-6B-shaped layer), `quantize`/`dequant` (GB/s of the offline
-steps), `e2e` (same metric through the host-buffer entry point, copies timed) and
-`cpu_baseline` (the numpy oracle timed on this host's cores on a bounded sample).
+(packed codes + scales + x + y bytes of a step) / step time.  Further keys: `roofline` (decode
+kernel against the measured HBM copy bandwidth), `sustained` (the same step launched back to back
+for more than a second, with the SM clock sampled inside the region and the rate binned by clock),
+`e2e` (the same metric through the host-buffer entry point, copies timed), `sweeps` (the M sweeps of
+the ChatGLM2-6B-shaped and the 14B-class stack: microseconds, GB/s, TFLOP/s and t_roof / t per
+point, with the bound named), `prefill`, `quantize`/`dequant`, the objects of the widened rows,
+`cpu_baseline` (the numpy oracle timed on this host's cores on a bounded sample) and, as the LAST
+key, `summary`: the few figures that matter, short enough to survive a truncated log.
 
-`--impl reference` times the CPU oracle instead (rank 0 only).
+`--impl reference` times the CPU oracle instead (rank 0 only).  `--gpus N` without a torchrun
+environment starts N ranks itself (one independent replica of the stack per GPU).
 """
 
 from __future__ import annotations
@@ -31,10 +35,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel on the default
-# workload (Gemma-2B-shaped stack, M = 1), from the ncu capture summarised in
-# profiles/gemv_decode_batch_gemma2b_m1.md; other workloads report null.
-DECODE_TRAFFIC_BYTES_GEMMA2B_M1 = 1.0599e9 + 7.3e6
+# dram__bytes_read.sum + dram__bytes_write.sum per LAYER of one launch of the decode list kernel at
+# M = 1, from the ncu captures summarised under profiles/ (gemv_decode_batch_*_m1.md).  The 14B-class
+# figure was captured on 8 of the 40 layers (a capture has to stay small) and is scaled by the layer
+# count: a launch's traffic is its weights, read once, so it grows in proportion.  Other workloads
+# report null.
+DECODE_TRAFFIC_BYTES_PER_LAYER_M1 = {"gemma2b": (1.0599e9 + 7.3e6) / 18, "llm14b": None}
 
 METRIC = "e0m4_decode_gemv_hbm_gbps"
 UNIT = "GB/s"
@@ -178,7 +184,7 @@ def workload_config(stack, layers, n_matrices, M, nbytes, world):
         "workload": f"{stack}-shaped decode stack: {layers} layers x {n_matrices} E0M4 matmuls, M={M}, group 128",
         "bytes_per_step": nbytes,
         "l2": "inputs larger than L2 (packed stack streamed per step)",
-        "launch": "tl_e0m4_matmul_batch over the whole stack (one persistent kernel per 128 "
+        "launch": "tl_e0m4_matmul_batch over the whole stack (one persistent kernel per 192 "
                   "independent problems), replayed as a CUDA graph",
         "parallelism": f"replicas x{world}",
     }
@@ -259,7 +265,7 @@ def make_call_step(binding, torch, problems, M, ws):
 
 
 def make_batch_step(binding, torch, problems, M, ws):
-    """One tl_e0m4_matmul_batch call for the whole stack (a persistent kernel per 128 problems)."""
+    """One tl_e0m4_matmul_batch call for the whole stack (a persistent kernel per 192 problems)."""
     import ctypes
 
     arr = binding.make_problem_array([(p["x"], p["packed"], p["scales"], p["y"]) for p in problems])
@@ -299,6 +305,22 @@ def time_events(torch, fn, iters):
     end.record()
     torch.cuda.synchronize()
     return start.elapsed_time(end) / iters  # ms per call
+
+
+def time_events_clocked(torch, fn, iters, index):
+    """time_events plus the SM clock read while the timed work is still in flight."""
+    sampler = ClockSampler(index)
+    start = torch.cuda.Event(enable_timing=True)
+    end = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record()
+    for _ in range(iters):
+        fn()
+    end.record()
+    clocks = sampler.stop()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / iters, clocks["sm_mhz"]
 
 
 def bench_prefill(binding, workloads, torch, dev, peaks, Ms=(128, 512, 2048)):
@@ -741,6 +763,178 @@ def bench_offline(binding, workloads, torch, dev):
             {"gbps": d_bytes / (d_ms * 1e-3) / 1e9, "ms": d_ms, "shape": [K, N]})
 
 
+def bench_m_sweep(binding, workloads, torch, dev, peaks, stack_name, tokens, layers=8):
+    """The M sweep of a configuration on `layers` layers of its stack (every layer has its own
+    weights, 0.9-1.3 GB in all, so nothing comes from L2).  Up to 128 tokens a point is measured
+    twice: as ONE tl_e0m4_matmul_batch call over all matrices (every matrix with its own
+    activations) and as one tl_e0m4_matmul call per matrix; above 128 tokens per call only (the
+    activations of a layer are then shared by all layers to bound memory).  Every leg is a CUDA
+    graph.  t_roof = max(bytes / measured HBM peak, flops / measured tensor peak); `bound` names the
+    larger of the two."""
+    spec = workloads.STACKS[stack_name]
+    mats = []
+    for layer in range(layers):
+        for name, K, N in spec["matrices"]:
+            w = workloads.weights_torch(K, N, workloads.seed_for("sweep", stack_name, layer, name), dev)
+            mats.append((K, N) + tuple(binding.tl_e0m4_quantize(w)))
+            del w
+    rows = []
+    for M in tokens:
+        own = M <= 128  # own activations per matrix (what a list call needs); shared per shape above
+        outl = 0.01 if M > 16 else 0.0
+        if own:
+            xs = [workloads.activations_torch(M, K, workloads.seed_for("sweep", "x", i), dev, outl)
+                  for i, (K, _, _, _) in enumerate(mats)]
+            ys = [torch.empty((M, N), dtype=torch.float16, device=dev) for _, N, _, _ in mats]
+        else:
+            xk = {K: workloads.activations_torch(M, K, workloads.seed_for("sweep", "x", K), dev, outl)
+                  for K, _, _, _ in mats}
+            yn = {N: torch.empty((M, N), dtype=torch.float16, device=dev) for _, N, _, _ in mats}
+            xs = [xk[K] for K, _, _, _ in mats]
+            ys = [yn[N] for _, N, _, _ in mats]
+        nbytes = sum(K * N * BYTES_PER_WEIGHT + 2 * M * (K + N) for K, N, _, _ in mats)
+        flops = sum(2.0 * M * K * N for K, N, _, _ in mats)
+        t_hbm, t_tc = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
+        t_roof = max(t_hbm, t_tc)
+        row = {"M": M, "bound": "hbm" if t_hbm >= t_tc else "tensor", "t_roof_us": t_roof * 1e6}
+        ws = binding.tl_e0m4_workspace(max([binding.tl_e0m4_matmul_batch_workspace()] +
+                                           [binding.tl_e0m4_matmul_workspace(M, K, N) for K, N, _, _ in mats]), dev)
+        legs = []
+        if own:
+            arr = binding.make_problem_array([(x, pk, sc, y) for (_, _, pk, sc), x, y in zip(mats, xs, ys)])
+            legs.append(("list", lambda: binding.tl_e0m4_matmul_batch(arr, M, ws)))
+
+        def per_call():
+            for (K, N, pk, sc), x, y in zip(mats, xs, ys):
+                binding.tl_e0m4_matmul(x, pk, sc, N, y=y, workspace=ws)
+
+        legs.append(("per_call", per_call))
+        for name, fn in legs:
+            graph, launches = capture(binding, torch, fn)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            time.sleep(0.1)  # let the power-cap controller forget the previous point
+            us, mhz = time_events_clocked(torch, graph.replay, 20 if M <= 256 else 5, dev.index or 0)
+            us *= 1e3
+            row[name] = {"us": us, "launches": launches, "gbps": nbytes / us / 1e3, "tflops": flops / us / 1e6,
+                         "t_roof_over_t": t_roof * 1e6 / us, "sm_mhz": mhz}
+            del graph
+        row["best"] = max(row[k]["t_roof_over_t"] for k, _ in legs)
+        rows.append(row)
+        del xs, ys, ws
+    return {"stack": stack_name, "layers": layers, "weight_bytes": sum(K * N * BYTES_PER_WEIGHT for K, N, _, _ in mats),
+            "points": rows}
+
+
+def run_sustained(torch, graph, nbytes, index, seconds=1.5, chunk_steps=None, ms_per_step=1.0):
+    """The headline step launched back to back for `seconds`, the SM clock sampled every 10 ms inside
+    the region.  The steps are timed in chunks (a CUDA event after each), every chunk gets the median of
+    the clock samples that fall into it (the host clock and the device time line are aligned at the first
+    record), and the rate is reported overall and per 50-MHz clock bin."""
+    chunk_steps = chunk_steps or max(1, int(round(50.0 / ms_per_step)))   # chunks of about 50 ms
+    chunks = max(4, int(seconds * 1e3 / (chunk_steps * ms_per_step)))
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(chunks + 1)]
+    samples = []
+    stop = threading.Event()
+    sampler = ClockSampler(index)
+
+    def poll(t0):
+        while not stop.is_set() and sampler.nv is not None:
+            try:
+                samples.append((time.perf_counter() - t0, sampler.nv.nvmlDeviceGetClockInfo(sampler.h, sampler.nv.NVML_CLOCK_SM)))
+                sampler._once()
+            except Exception:
+                break
+            stop.wait(0.01)
+
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    events[0].record()
+    thread = threading.Thread(target=poll, args=(t0,), daemon=True)
+    thread.start()
+    for c in range(chunks):
+        for _ in range(chunk_steps):
+            graph.replay()
+        events[c + 1].record()
+    torch.cuda.synchronize()
+    stop.set()
+    thread.join()
+    edges = [0.0] + [events[0].elapsed_time(e) * 1e-3 for e in events[1:]]
+    total_s = edges[-1]
+    bins = {}
+    for c in range(chunks):
+        inside = sorted(mhz for t, mhz in samples if edges[c] <= t < edges[c + 1])
+        if not inside:
+            continue
+        key = int(round(inside[len(inside) // 2] / 50.0) * 50)
+        b = bins.setdefault(key, [0.0, 0])
+        b[0] += edges[c + 1] - edges[c]
+        b[1] += chunk_steps
+    all_mhz = sorted(m for _, m in samples)
+    first = nbytes * chunk_steps / (edges[1] - edges[0]) / 1e9
+    last = nbytes * chunk_steps / (edges[-1] - edges[-2]) / 1e9
+    return {"value": nbytes * chunks * chunk_steps / total_s / 1e9, "unit": UNIT, "seconds": total_s,
+            "steps": chunks * chunk_steps, "first_chunk_gbps": first, "last_chunk_gbps": last,
+            "sm_mhz_median": all_mhz[len(all_mhz) // 2] if all_mhz else None, "sm_max_mhz": sampler.max_mhz,
+            "reasons": sorted(sampler.reasons), "clock_samples": len(all_mhz),
+            "gbps_by_sm_mhz": {str(k): nbytes * v[1] / v[0] / 1e9 for k, v in sorted(bins.items())}}
+
+
+def bench_launch_floor(binding, torch, dev):
+    """What a launch costs on this machine whatever the kernel does: the smallest problem the matmul
+    accepts (one tile: 128 x 16) launched back to back in one CUDA graph, each launch depending on
+    its predecessor through programmatic dependent launch as every launch of the library does."""
+    w = torch.zeros((128, 16), dtype=torch.float32, device=dev)
+    pk, sc = binding.tl_e0m4_quantize(w)
+    x = torch.zeros((1, 128), dtype=torch.float16, device=dev)
+    y = torch.empty((1, 16), dtype=torch.float16, device=dev)
+    ws = binding.tl_e0m4_workspace(binding.tl_e0m4_matmul_workspace(1, 128, 16), dev)
+    graph, _ = capture(binding, torch, lambda: [binding.tl_e0m4_matmul(x, pk, sc, 16, y=y, workspace=ws) for _ in range(100)])
+    graph.replay()
+    return {"one_tile_matmul_back_to_back_us": time_events(torch, graph.replay, 10) * 1e3 / 100}
+
+
+def _r(v, digits=4):
+    return None if v is None else round(float(v), digits)
+
+
+def make_summary(line, peaks):
+    """The figures that matter, in one short object printed as the LAST key of the line."""
+    out = {"workload": line["config"]["workload"], "value_gbps": _r(line["value"], 1),
+           "roofline_frac": _r(line["roofline"]["frac"]), "hbm_peak_gbs": peaks["hbm_gbs"],
+           "tensor_peak_tflops": peaks["bf16_tflops"],
+           "per_call_gbps": _r(line["per_call"]["value"], 1),
+           "per_call_frac": _r(line["per_call"]["value"] / line["n_gpus"] / peaks["hbm_gbs"]),
+           "e2e_one_stream_gbps": _r(line["e2e"]["value"], 1),
+           "e2e_two_streams_gbps": _r(line["e2e"]["two_streams"]["value"], 1),
+           "two_lanes_gbps": _r(line["two_lanes"]["value"], 1)}
+    if line.get("sustained"):
+        out["sustained_gbps"] = _r(line["sustained"]["value"], 1)
+        out["sustained_frac"] = _r(line["sustained"]["frac_of_measured_hbm"])
+        out["sustained_sm_mhz"] = line["sustained"]["sm_mhz_median"]
+    if "prefill" in line:
+        out["prefill_tflops"] = {k: _r(v["tflops"], 1) for k, v in line["prefill"].items() if k.startswith("M")}
+        out["prefill_frac_of_burst"] = {k: _r(v["frac_of_measured_bf16_burst"]) for k, v in line["prefill"].items()
+                                        if k.startswith("M")}
+    for name, sweep in line.get("sweeps", {}).items():
+        out["sweep_" + name] = {f"M{r['M']}": [r["bound"], _r(r["best"], 3)] for r in sweep["points"]}
+    if "decode_layer_chain" in line:
+        out["decode_layer_chain"] = {k: _r(v, 3) for k, v in line["decode_layer_chain"].items()
+                                     if k in ("us_per_layer", "t_roof_over_t", "chain_us_per_layer", "chain_t_roof_over_t")}
+    if "int4_twin" in line:
+        row = line["int4_twin"]["table1_m1_latency"][0]
+        floor = line.get("launch_floor", {}).get("one_tile_matmul_back_to_back_us")
+        t_roof = (row["K"] * row["N"] * BYTES_PER_WEIGHT + 2 * (row["K"] + row["N"])) / (peaks["hbm_gbs"] * 1e3)
+        out["config1_gemv_4096x4096_m1"] = {"us": _r(row["fp4_us"], 2), "frac_of_hbm_roofline": _r(t_roof / row["fp4_us"]),
+                                            "launch_floor_us": _r(floor, 2),
+                                            "frac_of_roofline_plus_launch_floor":
+                                                _r((t_roof + floor) / row["fp4_us"]) if floor else None}
+    if "cpu_baseline" in line:
+        out["cpu_oracle_gbps"] = _r(line["cpu_baseline"]["value"], 4)
+    return out
+
+
 def run_native(args):
     import torch
 
@@ -764,10 +958,18 @@ def run_native(args):
         dist.barrier()
     binding.lib()
     peaks = load_peaks()
-    if args.object == "e0m8":
-        # only the E0M8 object, at the token counts given by --M (a profiling aid: one JSON line)
+    if args.object:
+        # only one of the extra objects (a profiling aid: one JSON line); --M picks the token count where one applies
         if rank == 0:
-            print(json.dumps({"object": "e0m8", "e0m8": bench_e0m8(binding, workloads, torch, dev, peaks, (args.M,))}))
+            one = {"e0m8": lambda: bench_e0m8(binding, workloads, torch, dev, peaks, (args.M,)),
+                   "sweep": lambda: bench_m_sweep(binding, workloads, torch, dev, peaks, args.stack, (args.M,),
+                                                  layers=args.layers or 8),
+                   "list_sweep": lambda: bench_list_sweep(binding, workloads, torch, dev, peaks),
+                   "chain": lambda: bench_decode_layer_chain(binding, workloads, torch, dev, peaks),
+                   "prefill": lambda: bench_prefill(binding, workloads, torch, dev, peaks),
+                   "int4_twin": lambda: bench_int4_twin(binding, workloads, torch, dev, peaks),
+                   "launch_floor": lambda: bench_launch_floor(binding, torch, dev)}[args.object]()
+            print(json.dumps({"object": args.object, args.object: one}), flush=True)
         return
 
     spec = workloads.STACKS[args.stack]
@@ -780,7 +982,7 @@ def run_native(args):
     nbytes = step_bytes(spec["matrices"], layers, M)
     warm = max(args.warmup, 3)
 
-    # headline: the whole stack as one batch (one persistent kernel per 128 problems), replayed
+    # headline: the whole stack as one batch (one persistent kernel per 192 problems), replayed
     # as a CUDA graph
     batch_step, _arr = make_batch_step(binding, torch, problems, M, ws)
     graph, launches_per_step = capture(binding, torch, batch_step)
@@ -804,7 +1006,6 @@ def run_native(args):
     total_ms = replicas.max_over_ranks(start.elapsed_time(end), dist, dev)
     ms_per_step = total_ms / args.steps
     value = replicas.whole_job_throughput(nbytes, ms_per_step * 1e-3, world) / 1e9
-
     # the same stack as one tl_e0m4_matmul call per matrix (one kernel launch each), also a graph
     call_graph, call_launches = capture(binding, torch, make_call_step(binding, torch, problems, M, ws))
     for _ in range(warm):
@@ -886,7 +1087,7 @@ def run_native(args):
 
     extra = {}
     if rank == 0 and world == 1:
-        del problems, graph, call_graph, batch_step
+        del call_graph
         torch.cuda.empty_cache()
         if not args.no_prefill:
             extra["prefill"] = bench_prefill(binding, workloads, torch, dev, peaks)
@@ -895,6 +1096,13 @@ def run_native(args):
             extra["group_sizes"] = bench_group_sizes(binding, workloads, torch, dev, peaks)
             extra["e0m8"] = bench_e0m8(binding, workloads, torch, dev, peaks)
             extra["list_sweep"] = bench_list_sweep(binding, workloads, torch, dev, peaks)
+            extra["sweeps"] = {
+                "chatglm2_6b": bench_m_sweep(binding, workloads, torch, dev, peaks, "chatglm2_6b",
+                                             (1, 4, 16, 128, 512, 2048)),
+                "llm14b": bench_m_sweep(binding, workloads, torch, dev, peaks, "llm14b",
+                                        (1, 2, 4, 8, 16, 64, 256, 1024, 4096)),
+            }
+            extra["launch_floor"] = bench_launch_floor(binding, torch, dev)
             extra["decode_layer_chain"] = bench_decode_layer_chain(binding, workloads, torch, dev, peaks)
             extra["rmsnorm"] = bench_rmsnorm(binding, workloads, torch, dev, peaks)
             extra["matmul_add"] = bench_matmul_add(binding, workloads, torch, dev)
@@ -905,6 +1113,16 @@ def run_native(args):
             extra["cpu_baseline"] = {"value": cb_bytes * len(times) / sum(times) / 1e9, "unit": UNIT,
                                      "cores": host_threads(), "kind": "oracle", "sample": desc}
 
+    # Last, so that its heat does not colour the other objects: the headline step back to back for more
+    # than a second, i.e. what the power cap leaves of the burst figure.
+    sustained = None
+    if not args.no_sustained:
+        sustained = run_sustained(torch, graph, nbytes, local_rank, seconds=args.sustained_seconds,
+                                  ms_per_step=ms_per_step)
+        step_s = replicas.max_over_ranks(sustained["seconds"] / sustained["steps"], dist, dev)
+        sustained["value"] = replicas.whole_job_throughput(nbytes, step_s, world) / 1e9
+        sustained["frac_of_measured_hbm"] = sustained["value"] / world / peaks["hbm_gbs"]
+
     if rank == 0:
         achieved = value / world
         # which roofline bounds a step at this M: the weight bytes or the tensor-core rate
@@ -913,8 +1131,8 @@ def run_native(args):
         if nbytes / peaks["hbm_gbs"] >= flops / (peaks["bf16_tflops"] * 1e3):
             roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": achieved / peaks["hbm_gbs"],
-                        "traffic": (DECODE_TRAFFIC_BYTES_GEMMA2B_M1
-                                    if (args.stack, M, layers) == ("gemma2b", 1, 18) else None),
+                        "traffic": (DECODE_TRAFFIC_BYTES_PER_LAYER_M1[args.stack] * layers / launches_per_step
+                                    if M == 1 and DECODE_TRAFFIC_BYTES_PER_LAYER_M1.get(args.stack) else None),
                         "algorithmic_bytes_per_launch": nbytes / launches_per_step}
         else:
             tflops = flops / (ms_per_step * 1e-3) / 1e12
@@ -929,18 +1147,22 @@ def run_native(args):
             "config": dict(workload_config(args.stack, layers, len(spec["matrices"]), M, nbytes, world),
                            tokens_per_s_equivalent=world * M / (ms_per_step * 1e-3)),
             "roofline": roofline,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
-                    "issue": "tl_e0m4_matmul_batch_host on two streams in turn, own staging and scratch each",
-                    "single_stream": {"value": replicas.whole_job_throughput(nbytes, serial_ms * 1e-3, world) / 1e9,
-                                      "ms_per_step": serial_ms}},
+            # like `value`, one step at a time: copy x in, the list call, copy y out, on one stream
+            "e2e": {"value": replicas.whole_job_throughput(nbytes, serial_ms * 1e-3, world) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": serial_ms,
+                    "issue": "tl_e0m4_matmul_batch_host, one stream, one step at a time",
+                    "two_streams": {"value": e2e_value, "ms_per_step": e2e_ms,
+                                    "issue": "the same call on two streams in turn, own staging and scratch each: "
+                                             "a step's copies run under its neighbour's kernel"}},
             "two_lanes": two_lanes,
+            "sustained": sustained,
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
             "per_call": per_call,
         }
         line.update(extra)
-        print(json.dumps(line), flush=True)
+        line["summary"] = make_summary(line, peaks)
+        print(json.dumps(line, separators=(",", ":")), flush=True)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -952,18 +1174,46 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["native", "reference"], default="native")
-    ap.add_argument("--stack", default="gemma2b")
+    ap.add_argument("--stack", default="llm14b")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = the stack's own)")
     ap.add_argument("--M", type=int, default=1)
-    ap.add_argument("--object", choices=["e0m8"], default=None,
-                    help="run only this extra object (at --M tokens) and print it")
+    ap.add_argument("--object", default=None,
+                    choices=["e0m8", "sweep", "list_sweep", "chain", "prefill", "int4_twin", "launch_floor"],
+                    help="run only this extra object (at --M tokens where one applies) and print it")
     ap.add_argument("--no-prefill", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true")
+    ap.add_argument("--sustained-seconds", type=float, default=1.5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
     else:
+        if int(os.environ.get("WORLD_SIZE", "1")) != args.gpus:
+            raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={os.environ.get('WORLD_SIZE', '1')}: "
+                             "launch one rank per GPU (or run without a torchrun environment and let bench.py start them)")
         run_native(args)
+
+
+def spawn_ranks(n):
+    """`--gpus N` given to a plain `python bench.py`: start N ranks of this same command under
+    torch.distributed.run (one replica per GPU) and pass their exit code on.  Refuses loudly when
+    the box has fewer than N GPUs: a run must never report fewer GPUs than it was asked for."""
+    import socket
+    import subprocess
+
+    import torch
+
+    have = torch.cuda.device_count()
+    if have < n:
+        raise SystemExit(f"bench.py: --gpus {n} asked for, but this machine has {have} CUDA device(s)")
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 if __name__ == "__main__":

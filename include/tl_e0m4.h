@@ -213,8 +213,8 @@ size_t tl_e0m4_matmul_batch_workspace(void);
 /* Section 2.2, decoding stage and batched decoding: the same product for `count` INDEPENDENT
  * problems that share M (1 <= M <= 128; larger M is TL_ERR_SHAPE), e.g. the q/k/v projections of
  * one layer, gate and up, or a whole stack of layers whose inputs are all known.  All problems run
- * in one persistent kernel that streams their packed weights back to back (longer lists than 128
- * take one launch per 128): the register-fragment vector-matrix kernel up to 8 tokens, the
+ * in one persistent kernel that streams their packed weights back to back (longer lists than 192
+ * take one launch per 192): the register-fragment vector-matrix kernel up to 8 tokens, the
  * tensor-core kernel from 9 tokens on.  problems_host: HOST array of `count` descriptors; it is
  * read during the call only.  No problem may read what another problem of the same batch writes
  * (no y_dev may alias an x_dev or another y_dev).  The workspace follows the rules of

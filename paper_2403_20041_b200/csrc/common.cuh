@@ -78,7 +78,7 @@ struct DecodeProblem {
   bool swiglu = false;          // single-problem launches: y[M, N/2] = silu(gate) * up over column blocks of 8
   int64_t add_stride = -1;      // elements between the addend's token rows; -1 = N, 0 = one bias row for all tokens
 };
-constexpr int kMaxDecodeBatch = 128;  // problems per launch; longer lists take several launches
+constexpr int kMaxDecodeBatch = 192;  // problems per launch (the 160 matrices of a 40-layer stack fit one); longer lists take several
 size_t decode_workspace_bytes();
 cudaError_t launch_gemv_decode(const __half* x, const uint32_t* packed, const uint32_t* scales,
                                __half* y, int64_t M, int64_t K, int64_t N, void* workspace,

@@ -139,8 +139,13 @@ struct StageWalk {
   const DecodeParams<NB>& p;
   int j, panel, g, left, ng, panels;
   __device__ StageWalk(const DecodeParams<NB>& p_, int c0, int n_chunks) : p(p_), left(n_chunks) {
-    j = 0;
-    while (j + 1 < p.count && p.prob[j + 1].chunk_begin <= c0) ++j;
+    // the problem whose chunks contain c0: the last one that begins at or before it
+    int lo = 0, hi = p.count - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (p.prob[mid].chunk_begin <= c0) lo = mid; else hi = mid - 1;
+    }
+    j = lo;
     ng = p.prob[j].ng;
     panels = p.prob[j].panels;
     const int off = c0 - p.prob[j].chunk_begin;
