@@ -22,5 +22,6 @@ from .e0m4 import (  # noqa: F401
 )
 from .int4 import quantize_int4  # noqa: F401
 from .kvcache import kv_append  # noqa: F401
-from .norm import layernorm, rmsnorm  # noqa: F401
+from .norm import layernorm, rms_scale, rmsnorm  # noqa: F401
+from .chain import chain_step  # noqa: F401
 from .layout import pack, unpack, packed_sizes  # noqa: F401

@@ -143,14 +143,19 @@ def dequantize(codes, d_h, b_h, group: int = GROUP, n: int = 1, bits: int = 4):
     return out.astype(np.float16).reshape(K, N)
 
 
-def matmul(x_h, w_hat_h, addend_h=None):
+def matmul(x_h, w_hat_h, addend_h=None, row_scale=None):
     """Section 2.2: half-precision activation times dequantized weight,
     y[m, n] = sum_k x[m, k] * w_hat[k, n], here evaluated in double.  With `addend_h`
-    (fp16 [M, N]) the fused form of Section 2.2's operator fusion: the element-wise
-    residual add that follows the matmul, y + addend, still in double."""
+    (fp16 [M, N], or [N] for a bias row) the fused form of Section 2.2's operator fusion: the
+    element-wise add that follows the matmul, y + addend, still in double.  With `row_scale`
+    (double [M]) every row of the product is multiplied by its factor BEFORE the addend:
+    y[m, n] = row_scale[m] * sum_k x[m, k] w_hat[k, n] + addend[m, n]  (the rms-norm that precedes
+    a matmul, with its gain folded into the weights, is exactly such a factor: oracle.rms_scale)."""
     x = np.asarray(x_h, dtype=np.float16).astype(np.float64)
     w = np.asarray(w_hat_h, dtype=np.float16).astype(np.float64)
     y = x @ w
+    if row_scale is not None:
+        y = y * np.asarray(row_scale, dtype=np.float64).reshape(-1, 1)
     if addend_h is not None:
         y = y + np.asarray(addend_h, dtype=np.float16).astype(np.float64)
     return y

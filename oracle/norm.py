@@ -32,6 +32,14 @@ def rmsnorm(x_h, gamma_h, eps: float, residual_h=None):
     return y if s_h is None else (y, s_h)
 
 
+def rms_scale(x_h, eps: float):
+    """The row factor of the rms-norm alone: r[m] = 1 / sqrt(mean_k(x[m, :]^2) + eps), double [M].
+    rmsnorm(x, gamma) = x * r * gamma; with gamma folded into the weights of the matmul that
+    follows, (x * r * gamma) . W = r * (x . (gamma * W)): the norm becomes a factor per output row."""
+    x = np.asarray(x_h, dtype=np.float16).astype(np.float64)
+    return 1.0 / np.sqrt((x * x).mean(axis=1) + float(eps))
+
+
 def layernorm(x_h, gamma_h, beta_h, eps: float, residual_h=None):
     """x_h [M, K] fp16, gamma_h / beta_h [K] fp16 -> y fp16 [M, K]  (and s fp16 [M, K] with a residual)."""
     x = np.asarray(x_h, dtype=np.float16).astype(np.float64)
