@@ -233,6 +233,57 @@ tl_status tl_e0m4_matmul_batch_host(const tl_e0m4_problem* problems_host, int co
                                     void* y_host, const void* y_stage_dev, size_t y_bytes,
                                     void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* One step of a decode chain: a matmul of tl_e0m4_matmul with the element-wise operators around it
+ * fused in (Section 2.2, operator fusions), as one descriptor. */
+typedef enum {
+  TL_EPILOGUE_NONE = 0,   /* y[M, N] = Y                                                     */
+  TL_EPILOGUE_ADD = 1,    /* y[M, N] = Y + addend[M, N]   (addend_dev may be y_dev)          */
+  TL_EPILOGUE_BIAS = 2,   /* y[M, N] = Y + bias[N]                                            */
+  TL_EPILOGUE_SWIGLU = 3  /* y[M, N / 2] = silu(gate) * up over column blocks of eight of Y,
+                             as tl_e0m4_matmul_swiglu                                        */
+} tl_epilogue;
+
+typedef struct tl_e0m4_step {
+  const void* x_dev;       /* fp16 [M, K] row-major */
+  const void* packed_dev;  /* packed codes of W[K, N] */
+  const void* scales_dev;  /* scale words of W[K, N] */
+  void* y_dev;             /* fp16 [M, N] ([M, N / 2] with TL_EPILOGUE_SWIGLU), fully overwritten */
+  const void* addend_dev;  /* fp16 [M, N] (ADD) or [N] (BIAS), else NULL */
+  int64_t K;
+  int64_t N;
+  int32_t epilogue;        /* a tl_epilogue */
+  int32_t after_previous;  /* non-zero: this step reads (x_dev, addend_dev) or overwrites what an EARLIER step of
+                              the list writes, so it begins only when all earlier steps are complete;
+                              zero: it is independent of every step since the last such barrier */
+  int32_t rms_scale;       /* non-zero: Y is x . W with every row multiplied by 1 / sqrt(mean_k x[m, k]^2 + rms_eps):
+                              the rms-norm that precedes the matmul, its gain folded into W by the caller
+                              (quantize diag(gamma) . W) */
+  float rms_eps;
+} tl_e0m4_step;
+
+/* Bytes of device scratch tl_e0m4_matmul_chain needs (a constant, about 2.7 MB).  Host only. */
+size_t tl_e0m4_matmul_chain_workspace(void);
+
+/* Section 2.2, the decoding stage as a model runs it: a sequence of matmuls in which one consumes
+ * what another produces (norm -> qkv + bias -> ... -> o + residual -> norm -> gate_up + SwiGLU ->
+ * down + residual, layer after layer).  Y = x . W (fp32 accumulation), optionally scaled per row
+ * (rms_scale), then the epilogue, rounded once to fp16.  1 <= M <= 8 (TL_ERR_SHAPE above; batches
+ * of more tokens take one tl_e0m4_matmul call per step).
+ * All steps run in ONE persistent kernel per 128 steps.  Steps are processed in list order by all
+ * CTAs together; where a step has after_previous set, the kernel waits (on the device, per CTA,
+ * only for the activations: the packed weights of later steps keep streaming into shared memory
+ * meanwhile) until every earlier step is complete.  Steps without it run as the problems of
+ * tl_e0m4_matmul_batch do and must be independent of the steps since the last barrier.
+ * steps_host: HOST array, read during the call only.  Weights must be complete before the kernel
+ * preceding this call on the stream starts (see tl_e0m4_matmul).  The workspace
+ * (tl_e0m4_matmul_chain_workspace() bytes) follows the rules of tl_e0m4_workspace_init.
+ * The kernel's CTAs wait for one another, so all of them must be resident at once: the launch is
+ * sized to fit an otherwise idle GPU, and a call should not share the GPU with another long-running
+ * kernel (every wait is bounded: if the grid cannot become resident within about two seconds the
+ * call ends with TL_ERR_TIMEOUT in the status word instead of hanging). */
+tl_status tl_e0m4_matmul_chain(const tl_e0m4_step* steps_host, int count, int64_t M, int group,
+                               void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* (No counterpart in the paper: this entry point exists for deployment reasons only.)
  * The decoding product of tl_e0m4_matmul for callers that cannot obtain device memory at the
  * time of the call and therefore have no workspace to pass: code running between the

@@ -49,6 +49,8 @@ SYMBOLS = {
     "tl_e0m4_matmul_batch_workspace": (_sz, []),
     "tl_e0m4_matmul_batch": (_int, [_vp, _int, _i64, _int, _vp, _sz, _vp]),
     "tl_e0m4_matmul_batch_host": (_int, [_vp, _int, _i64, _int, _vp, _vp, _sz, _vp, _vp, _sz, _vp, _sz, _vp]),
+    "tl_e0m4_matmul_chain_workspace": (_sz, []),
+    "tl_e0m4_matmul_chain": (_int, [_vp, _int, _i64, _int, _vp, _sz, _vp]),
     "tl_e0m4_matmul_noalloc": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp]),
     "tl_e0m4_matmul_noalloc_scratch_bytes": (_sz, []),
     "tl_e0m4_matmul_host_staging": (_sz, [_i64, _i64, _i64]),
@@ -74,6 +76,17 @@ class Problem(ctypes.Structure):
     _fields_ = [("x_dev", _vp), ("packed_dev", _vp), ("scales_dev", _vp), ("y_dev", _vp),
                 ("K", _i64), ("N", _i64)]
 
+
+class Step(ctypes.Structure):
+    """Mirror of the C struct tl_e0m4_step."""
+
+    _fields_ = [("x_dev", _vp), ("packed_dev", _vp), ("scales_dev", _vp), ("y_dev", _vp), ("addend_dev", _vp),
+                ("K", _i64), ("N", _i64), ("epilogue", ctypes.c_int32), ("after_previous", ctypes.c_int32),
+                ("rms_scale", ctypes.c_int32), ("rms_eps", ctypes.c_float)]
+
+
+TL_EPILOGUE_NONE, TL_EPILOGUE_ADD, TL_EPILOGUE_BIAS, TL_EPILOGUE_SWIGLU = 0, 1, 2, 3
+_EPILOGUES = {"none": 0, "add": 1, "bias": 2, "swiglu": 3}
 
 _lib = None
 
@@ -477,6 +490,38 @@ def tl_e0m4_matmul_batch_host(problems, M: int, x_host, x_stage, y_host, y_stage
         x_stage.numel() * x_stage.element_size(), y_host.data_ptr(), _dev_ptr(y_stage, "y_stage"),
         y_stage.numel() * y_stage.element_size(), _dev_ptr(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), _stream(stream)), "tl_e0m4_matmul_batch_host")
+
+
+def tl_e0m4_matmul_chain_workspace() -> int:
+    return lib().tl_e0m4_matmul_chain_workspace()
+
+
+def make_step_array(steps):
+    """ctypes array of tl_e0m4_step from dicts with the keys x, packed, scales, y (CUDA tensors) and,
+    optionally, epilogue ("none", "add", "bias", "swiglu"), addend (CUDA tensor), after_previous (bool),
+    rms_eps (float or None)."""
+    arr = (Step * len(steps))()
+    for i, st in enumerate(steps):
+        x, y = st["x"], st["y"]
+        epi = _EPILOGUES[st.get("epilogue", "none")]
+        addend = st.get("addend")
+        N = y.shape[1] * (2 if epi == TL_EPILOGUE_SWIGLU else 1)
+        eps = st.get("rms_eps")
+        arr[i] = Step(_dev_ptr(x, "x"), _dev_ptr(st["packed"], "packed"), _dev_ptr(st["scales"], "scales"),
+                      _dev_ptr(y, "y"), _dev_ptr(addend, "addend") if addend is not None else None,
+                      x.shape[1], N, epi, 1 if st.get("after_previous") else 0, 0 if eps is None else 1,
+                      0.0 if eps is None else float(eps))
+    return arr
+
+
+def tl_e0m4_matmul_chain(steps, M: int, workspace, group: int = GROUP, stream=None):
+    """Runs a list of decode steps (M <= 8), some of which consume what earlier ones produce, in one
+    persistent launch per 128 steps.  `steps` is a list of dicts (see make_step_array) or an array
+    built by it."""
+    arr = steps if isinstance(steps, ctypes.Array) else make_step_array(steps)
+    _check(lib().tl_e0m4_matmul_chain(ctypes.cast(arr, _vp), len(arr), M, group, _dev_ptr(workspace, "workspace"),
+                                      workspace.numel() * workspace.element_size(), _stream(stream)),
+           "tl_e0m4_matmul_chain")
 
 
 def tl_e0m4_matmul_noalloc(x, packed, scales, y, group: int = GROUP, stream=None):

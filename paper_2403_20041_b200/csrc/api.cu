@@ -1,6 +1,7 @@
 // extern "C" boundary: argument validation, the M-based dispatcher and the host-buffer variant.
 #include <atomic>
 #include <cstring>
+#include <vector>
 
 #include "common.cuh"
 #include "tuning.h"
@@ -389,6 +390,48 @@ tl_status tl_e0m4_matmul_swiglu(const void* x_dev, const void* packed_dev, const
                                 void* workspace_dev, size_t workspace_bytes, void* stream) {
   return matmul_any(x_dev, packed_dev, scales_dev, nullptr, true, y_dev, M, K, N, group, workspace_dev,
                     workspace_bytes, stream);
+}
+
+size_t tl_e0m4_matmul_chain_workspace(void) { return decode_chain_workspace_bytes(); }
+
+tl_status tl_e0m4_matmul_chain(const tl_e0m4_step* steps_host, int count, int64_t M, int group,
+                               void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (!steps_host || !workspace_dev) return TL_ERR_NULL;
+  if (count <= 0 || count > 65536) return TL_ERR_SHAPE;
+  if (M <= 0 || M > kRegisterMaxM) return TL_ERR_SHAPE;
+  std::vector<ChainStep> steps((size_t)count);
+  for (int j = 0; j < count; ++j) {
+    const tl_e0m4_step& q = steps_host[j];
+    if (!q.x_dev || !q.packed_dev || !q.scales_dev || !q.y_dev) return TL_ERR_NULL;
+    const tl_status st = check_shape(q.K, q.N, group);
+    if (st != TL_OK) return st;
+    if (q.epilogue < TL_EPILOGUE_NONE || q.epilogue > TL_EPILOGUE_SWIGLU) return TL_ERR_SHAPE;
+    const bool wants_addend = q.epilogue == TL_EPILOGUE_ADD || q.epilogue == TL_EPILOGUE_BIAS;
+    if (wants_addend && !q.addend_dev) return TL_ERR_NULL;
+    if (q.rms_scale && !(q.rms_eps >= 0.0f)) return TL_ERR_SHAPE;
+    if (!aligned16(q.x_dev) || !aligned16(q.packed_dev) || !aligned16(q.scales_dev) || !aligned16(q.y_dev) ||
+        (wants_addend && !aligned16(q.addend_dev)))
+      return TL_ERR_ALIGN;
+    ChainStep& c = steps[(size_t)j];
+    c.x = static_cast<const __half*>(q.x_dev);
+    c.packed = static_cast<const uint32_t*>(q.packed_dev);
+    c.scales = static_cast<const uint32_t*>(q.scales_dev);
+    c.y = static_cast<__half*>(q.y_dev);
+    c.add = wants_addend ? static_cast<const __half*>(q.addend_dev) : nullptr;
+    c.add_stride = q.epilogue == TL_EPILOGUE_ADD ? q.N : 0;
+    c.K = q.K;
+    c.N = q.N;
+    c.epi = wants_addend ? 1 : (q.epilogue == TL_EPILOGUE_SWIGLU ? 2 : 0);
+    c.after_previous = q.after_previous != 0;
+    c.rms_eps = q.rms_scale ? q.rms_eps : -1.0f;
+  }
+  if (!aligned16(workspace_dev)) return TL_ERR_ALIGN;
+  if (workspace_bytes < decode_chain_workspace_bytes()) return TL_ERR_WORKSPACE;
+  const tl_status st = check_device();
+  if (st != TL_OK) return st;
+  const cudaError_t e =
+      launch_gemv_decode_chain(steps.data(), count, (int)M, workspace_dev, static_cast<cudaStream_t>(stream), group);
+  return e == cudaSuccess ? TL_OK : TL_ERR_CUDA;
 }
 
 tl_status tl_e0m4_matmul_noalloc(const void* x_dev, const void* packed_dev, const void* scales_dev,

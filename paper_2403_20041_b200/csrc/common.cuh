@@ -86,6 +86,26 @@ cudaError_t launch_gemv_decode(const __half* x, const uint32_t* packed, const ui
                                int group = kGroup, int64_t add_stride = -1);
 cudaError_t launch_gemv_decode_batch(const DecodeProblem* probs, int count, int M, void* workspace,
                                      cudaStream_t stream, int group = kGroup);
+// A chain of decode steps (M <= 8) in one persistent launch per 128 steps: a step with
+// `after_previous` set starts only when all earlier steps are complete, the others stream together
+// with their predecessor.  epi: 0 plain, 1 addend (add_stride N: a matrix, 0: a bias row), 2 SwiGLU.
+// rms_eps >= 0: every output row is scaled by rsqrt(mean_k x[m, k]^2 + eps) before the epilogue.
+// `workspace` holds decode_chain_workspace_bytes() bytes, zero on entry and left zero.
+struct ChainStep {
+  const __half* x;
+  const uint32_t* packed;
+  const uint32_t* scales;
+  __half* y;
+  const __half* add;
+  int64_t add_stride;
+  int64_t K, N;
+  int epi;
+  bool after_previous;
+  float rms_eps;
+};
+size_t decode_chain_workspace_bytes();
+cudaError_t launch_gemv_decode_chain(const ChainStep* steps, int count, int M, void* workspace, cudaStream_t stream,
+                                     int group = kGroup);
 // Decode launch that uses the library's own file-scope scratch array instead of a workspace.
 size_t builtin_scratch_bytes();
 cudaError_t launch_gemv_decode_builtin(const __half* x, const uint32_t* packed, const uint32_t* scales,

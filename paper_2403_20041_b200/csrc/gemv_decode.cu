@@ -28,6 +28,7 @@
 //     prefetches weights (which no predecessor writes) before it waits for its predecessor;
 //     activations, outputs and scratch are touched only after that wait.
 #include <atomic>
+#include <mutex>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -70,6 +71,7 @@ struct Prob {
 
 template <int NB>
 struct DecodeParams {
+  static constexpr bool kChain = false;
   uint8_t* ws;            // kMaxSlots slots of {fp32 [128][16] partial sums, chunk counter}, zero between calls
   unsigned int* status;   // device status word (0 = fine)
   int M;
@@ -86,6 +88,74 @@ struct DecodeParams {
   long long wait_limit;   // SM cycles after which a bounded wait gives up
   int skip_copies;        // diagnostics: the producer issues nothing, so every wait runs out
 };
+
+// ---- a chain of steps that may depend on one another (tl_e0m4_matmul_chain)
+// The steps are grouped into phases: a phase is a run of steps that do not read what another step
+// of the same phase writes, and every phase after the first begins only when ALL earlier steps are
+// complete.  Within a phase the chunk sequences of its steps are concatenated and cut over ALL CTAs
+// of the launch, exactly as a list of independent problems is; the CTAs walk the phases in order.
+// What crosses a phase boundary without waiting is the weight stream: a CTA's producer fills its
+// ring with the next phase's codes while the last CTAs are still finishing the current one.
+struct ChainProb {
+  const __half* x;
+  const uint8_t* packed;
+  const uint8_t* scales;
+  __half* y;
+  const __half* add;      // epi 1: fp16 addend, matrix (add_stride = N) or bias row (add_stride = 0)
+  long long add_stride;
+  int K, N, ng, nbs, panels;
+  int chunk_begin;        // first chunk of this step in its PHASE's concatenated sequence
+  int epi;                // 0 plain store, 1 addend, 2 SwiGLU over column blocks of 8
+  int phase;
+  float rms_eps;          // >= 0: every output row is multiplied by rsqrt(mean_k x[m, k]^2 + eps); < 0: no factor
+};
+
+struct ChainPhase {
+  int first, last;        // steps [first, last) of the launch
+  int chunks;             // chunks of the phase
+  int unit;               // as DecodeParams::unit, for this phase
+  unsigned int wait_target;  // panels of all earlier phases: the phase's activations exist once that many are final
+};
+
+constexpr int kMaxChain = 128;       // steps per launch (their descriptors travel as kernel parameters)
+constexpr int kChainRmsSlots = 8;    // row factors are kept for this many steps (a ring: consumers lag the row-sum warp by less)
+
+struct ChainParams {
+  static constexpr bool kChain = true;
+  uint8_t* ws;            // the scratch slots of DecodeParams::ws
+  unsigned int* status;
+  unsigned int* sync;     // [0] panels made final so far in this launch, [1] CTAs that have finished; zero between launches
+  int M;
+  int count;
+  int phases;
+  int stages;
+  int stage_bytes;
+  int xsum_offset;
+  long long wait_limit;
+  int skip_copies;
+  ChainProb prob[kMaxChain];
+  ChainPhase phase[kMaxChain];
+};
+
+// This CTA's contiguous range [c0, c1) of a sequence of `total` chunks.  unit > 0: equal ranges in
+// multiples of `unit` chunks; unit < 0: -unit CTAs per panel of a lone problem with `ng` groups and
+// `panels` panels, CTA i of a panel taking groups [ng i / s, ng (i + 1) / s).
+__device__ __forceinline__ void cta_range(int total, int unit, int ng, int panels, int& c0, int& c1) {
+  if (unit < 0) {
+    const int s = -unit;
+    const int panel = blockIdx.x / s, i = blockIdx.x - panel * s;
+    if (panel >= panels) {
+      c0 = c1 = 0;
+      return;
+    }
+    c0 = panel * ng + ng * i / s;
+    c1 = panel * ng + ng * (i + 1) / s;
+  } else {
+    const long long units = total / unit;
+    c0 = (int)(units * blockIdx.x / gridDim.x) * unit;
+    c1 = (int)(units * (blockIdx.x + 1) / gridDim.x) * unit;
+  }
+}
 
 // silu(g) * u in fp32 (Section 2.2's element-wise fusion for gated MLPs)
 __device__ __forceinline__ float swiglu(float g, float u) { return g / (1.0f + __expf(-g)) * u; }
@@ -134,13 +204,15 @@ constexpr uint32_t kMaskHi = 0x00F000F0u, kExpHi = 0x48004800u;  // 8 + code/8
 constexpr float kOffLo = 126.0f, kOffHi = 6.0f;
 
 // Walks the CTA's chunk range stage by stage, across problems: a stage never crosses a panel end.
-template <int NB>
+// For a chain the walk goes on through the phases: when the CTA's range of one phase is used up it
+// moves to the CTA's range of the next phase in which it has any chunks.
+template <class PT>
 struct StageWalk {
-  const DecodeParams<NB>& p;
+  const PT& p;
   int j, panel, g, left, ng, panels;
-  __device__ StageWalk(const DecodeParams<NB>& p_, int c0, int n_chunks) : p(p_), left(n_chunks) {
-    // the problem whose chunks contain c0: the last one that begins at or before it
-    int lo = 0, hi = p.count - 1;
+  int ph;  // chain: the phase being walked
+  __device__ void seek(int c0, int n_chunks, int lo, int hi) {
+    // the problem whose chunks contain c0: the last one of [lo, hi] that begins at or before it
     while (lo < hi) {
       const int mid = (lo + hi + 1) >> 1;
       if (p.prob[mid].chunk_begin <= c0) lo = mid; else hi = mid - 1;
@@ -151,7 +223,26 @@ struct StageWalk {
     const int off = c0 - p.prob[j].chunk_begin;
     panel = off / ng;
     g = off - panel * ng;
+    left = n_chunks;
   }
+  __device__ void next_phase() {
+    if constexpr (PT::kChain) {
+      left = 0;
+      while (++ph < p.phases) {
+        const ChainPhase& f = p.phase[ph];
+        int c0, c1;
+        cta_range(f.chunks, f.unit, p.prob[f.first].ng, p.prob[f.first].panels, c0, c1);
+        if (c1 > c0) {
+          seek(c0, c1 - c0, f.first, f.last - 1);
+          return;
+        }
+      }
+    }
+  }
+  // a list of independent problems: the range [c0, c0 + n_chunks) of the one sequence
+  __device__ StageWalk(const PT& p_, int c0, int n_chunks) : p(p_), ph(0) { seek(c0, n_chunks, 0, p.count - 1); }
+  // a chain: from the first phase on
+  __device__ explicit StageWalk(const PT& p_) : p(p_), j(0), panel(0), g(0), left(0), ng(1), panels(1), ph(-1) { next_phase(); }
   __device__ bool done() const { return left <= 0; }
   __device__ int groups() const {
     int n = ng - g;
@@ -171,6 +262,7 @@ struct StageWalk {
         panels = p.prob[j].panels;
       }
     }
+    if (PT::kChain && left <= 0) next_phase();
   }
 };
 
@@ -187,9 +279,11 @@ struct StageWalk {
 // with the k a tensor-core step covers (it takes 8 k from each 32-wide slice of the tile row), so
 // there every lane dequantizes its own slice — which lies in ONE group — to fp16 in registers,
 // (w1 - b) * d exactly as the standalone dequantizer does, and the sums need no correction.
-template <int MT, int NB, bool ROT, int EPI, int G>
+// PT: DecodeParams<NB> (a list of independent problems) or ChainParams (steps in phases, see above).
+template <int MT, class PT, bool ROT, int EPI, int G>
 __global__ void __launch_bounds__(kThreads, 2)
-gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
+gemv_decode_kernel(const __grid_constant__ PT p) {
+  constexpr bool CHAIN = PT::kChain;
   constexpr int kTileScaleBytes = tile_scale_bytes(G);
   constexpr int kXOffset = x_offset(G);
   extern __shared__ uint8_t smem_raw[];
@@ -198,6 +292,9 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)p.stages * p.stage_bytes);
   volatile int* flags = reinterpret_cast<volatile int*>(bars + 3 * kMaxStages);
   const uint32_t zero_block = ptx::smem_u32(bars + 3 * kMaxStages + 2);  // 64 zero bytes
+  // chain: row factors of the last kChainRmsSlots steps, [slot][8 tokens], and the step each slot holds
+  float* rms_val = reinterpret_cast<float*>(bars + 3 * kMaxStages + 10);
+  volatile int* rms_step = reinterpret_cast<volatile int*>(rms_val + kChainRmsSlots * 8);
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -217,32 +314,29 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
     ptx::fence_mbar_init();
   }
   if (tid < 16) reinterpret_cast<uint32_t*>(bars + 3 * kMaxStages + 2)[tid] = 0u;
+  if (CHAIN && tid < kChainRmsSlots) rms_step[tid] = -1;
   __syncthreads();
   ptx::pdl_launch_dependents();
 
-  // this CTA's contiguous range of chunks
-  int c0, c1;
-  if (p.unit < 0) {
-    // lone problem, -unit CTAs per panel: CTA i of a panel takes groups [ng i / s, ng (i + 1) / s)
-    const int s = -p.unit, ng = p.prob[0].ng;
-    const int panel = blockIdx.x / s, i = blockIdx.x - panel * s;
-    c0 = panel * ng + ng * i / s;
-    c1 = panel * ng + ng * (i + 1) / s;
-  } else {
-    const long long units = p.total_chunks / p.unit;
-    c0 = (int)(units * blockIdx.x / gridDim.x) * p.unit;
-    c1 = (int)(units * (blockIdx.x + 1) / gridDim.x) * p.unit;
+  // this CTA's contiguous range of chunks (a chain has one per phase: see StageWalk)
+  int c0 = 0, c1 = 0;
+  if constexpr (!CHAIN) {
+    cta_range(p.total_chunks, p.unit, p.prob[0].ng, p.prob[0].panels, c0, c1);
+    if (c1 <= c0) return;
   }
   const int n_chunks = c1 - c0;
-  if (n_chunks <= 0) return;
   const int M = p.M;
+  // one walk per warp role; all roles of a CTA walk the same stages in the same order
+  auto make_walk = [&]() {
+    if constexpr (CHAIN) return StageWalk<PT>(p); else return StageWalk<PT>(p, c0, n_chunks);
+  };
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------------- producer
     if (lane != 0 || p.skip_copies) return;
     const uint32_t ring_s = ptx::smem_u32(ring);
-    auto issue_w = [&](const StageWalk<NB>& w, int s) {
-      const Prob& q = p.prob[w.j];
+    auto issue_w = [&](const StageWalk<PT>& w, int s) {
+      const auto& q = p.prob[w.j];
       const int rest = q.nbs - kPanelTiles * w.panel;
       const int R = rest < kPanelTiles ? rest : kPanelTiles;
       const int tiles = w.groups() * R;
@@ -253,8 +347,8 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
       ptx::bulk_g2s(st, q.packed + tile0 * kTileBytes, tiles * kTileBytes, bar);
       ptx::bulk_g2s(st + kScaleOffset, q.scales + tile0 * kTileScaleBytes, tiles * kTileScaleBytes, bar);
     };
-    auto issue_x = [&](const StageWalk<NB>& w, int s) {
-      const Prob& q = p.prob[w.j];
+    auto issue_x = [&](const StageWalk<PT>& w, int s) {
+      const auto& q = p.prob[w.j];
       const uint32_t st = ring_s + s * p.stage_bytes + kXOffset;
       const uint32_t bar = xbar0 + 8 * s;
       const uint32_t bytes = w.groups() * 256;
@@ -263,9 +357,63 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
         ptx::bulk_g2s(st + m * kXRowBytes, q.x + (size_t)m * q.K + (size_t)w.g * kGroup, bytes, bar);
     };
 
+    if constexpr (CHAIN) {
+      // One thread, two cursors over the same walk.  The weight cursor runs ahead: it refills a stage
+      // as soon as the consumers release it, whatever phase the stage belongs to, so the codes of
+      // the next phase stream in while the current one is being finished.  The activation cursor
+      // follows: the slice of a stage is requested once its stage holds the weights AND every
+      // earlier phase is complete (the counter of final panels has reached the phase's target),
+      // because the slice is some earlier step's output.  Neither cursor blocks the other: both
+      // conditions are probed without waiting.
+      StageWalk<PT> w = make_walk();
+      StageWalk<PT> wx = w;
+      int iw = 0, ix = 0;            // stages whose weights / activations have been requested
+      int sw = 0, pw = 0, sx = 0;    // ring positions; pw: parity of the release the weight cursor needs next
+      unsigned int seen = 0;         // final panels observed so far
+      bool synced = false;           // pdl_wait done (before the first activation request)
+      long long t0 = clock64();
+      while (!wx.done()) {
+        bool progress = false;
+        if (!w.done() && (iw < S || ptx::mbar_test_wait(empty0 + 8 * sw, pw))) {
+          issue_w(w, sw);
+          w.next();
+          ++iw;
+          if (++sw == S) {
+            sw = 0;
+            if (iw > S) pw ^= 1;
+          }
+          progress = true;
+        }
+        if (ix < iw) {
+          if (!synced) {
+            ptx::pdl_wait();
+            synced = true;
+          }
+          const unsigned int target = p.phase[wx.ph].wait_target;
+          if (seen < target) {
+            seen = ptx::ld_acquire_gpu(p.sync);
+            if (seen >= target) ptx::fence_proxy_async_all();
+          }
+          if (seen >= target) {
+            issue_x(wx, sx);
+            wx.next();
+            ++ix;
+            if (++sx == S) sx = 0;
+            progress = true;
+          }
+        }
+        if (progress) {
+          t0 = clock64();
+        } else if (clock64() - t0 > p.wait_limit) {
+          atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
+          return;
+        }
+      }
+      return;
+    }
     // weights and scales of the first stages do not depend on the previous kernel
-    StageWalk<NB> w(p, c0, n_chunks);
-    StageWalk<NB> wx = w;
+    StageWalk<PT> w = make_walk();
+    StageWalk<PT> wx = w;
     int issued = 0;
     for (; issued < S && !w.done(); ++issued) {
       issue_w(w, issued);
@@ -301,7 +449,8 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
     static_assert(kStageGroups == 4, "the row-sum warp gives 8 lanes to each group of a stage");
     const int sub = lane >> 3, part = lane & 7;  // group of the stage, 16-halves slice of its 128 k
     const uint32_t ring_h = ptx::smem_u32(ring);
-    for (StageWalk<NB> w(p, c0, n_chunks); !w.done(); w.next()) {
+    [[maybe_unused]] int rms_last = -1;  // chain: the step whose row factors were formed last
+    for (StageWalk<PT> w = make_walk(); !w.done(); w.next()) {
       if (!ptx::mbar_wait_bounded(xbar0 + 8 * s, phase, p.wait_limit)) {
         if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
         return;
@@ -342,6 +491,41 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
         s = 0;
         phase ^= 1;
       }
+      if constexpr (CHAIN) {
+        // The first stage of a step with a folded rms-norm: the row factor rsqrt(mean x^2 + eps) of
+        // every token, from the whole activation row in global memory (L2: the row may have been
+        // written by other SMs a moment ago).  The consumers need it only when a panel ends, so it
+        // is formed after the stage has been handed over.
+        if (w.j != rms_last) {
+          rms_last = w.j;
+          const ChainProb& q = p.prob[w.j];
+          if (q.rms_eps >= 0.0f) {
+            (void)ptx::ld_acquire_gpu(p.sync);  // the row is final: the phase's activations were requested already
+            const int slot = w.j & (kChainRmsSlots - 1);
+            for (int m = 0; m < M; ++m) {
+              const uint4* row = reinterpret_cast<const uint4*>(q.x + (size_t)m * q.K);
+              float ss = 0.0f;
+              for (int i = lane; i < q.K / 8; i += 32) {
+                const uint4 v = __ldcg(row + i);
+                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+                const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&v.z));
+                const float2 f3 = __half22float2(*reinterpret_cast<const __half2*>(&v.w));
+                ss += (f0.x * f0.x + f0.y * f0.y) + (f1.x * f1.x + f1.y * f1.y) + (f2.x * f2.x + f2.y * f2.y) +
+                      (f3.x * f3.x + f3.y * f3.y);
+              }
+#pragma unroll
+              for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, off);
+              if (lane == 0) rms_val[slot * 8 + m] = rsqrtf(ss / (float)q.K + q.rms_eps);
+            }
+            __syncwarp();
+            if (lane == 0) {
+              __threadfence_block();
+              rms_step[slot] = w.j;
+            }
+          }
+        }
+      }
     }
     return;
   }
@@ -380,11 +564,11 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
   for (int v = 0; v < 4; ++v) chunk_off[v] = ((v + (rot ? 1 : 0)) & 3) * 16;
   const uint32_t ring_u32 = ptx::smem_u32(ring);
 
-  StageWalk<NB> w(p, c0, n_chunks);
+  StageWalk<PT> w = make_walk();
   int g_begin = w.g;
   int s = 0, phase = 0;
   while (!w.done()) {
-    const Prob& q = p.prob[w.j];
+    const auto& q = p.prob[w.j];
     const int rest = q.nbs - kPanelTiles * w.panel;
     const int R = rest < kPanelTiles ? rest : kPanelTiles;
     const int groups = w.groups();
@@ -510,9 +694,11 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
     const int panel = w.panel;
     const int ng = w.ng;
     const int g_end = w.g + groups;
+    const bool range_ends = w.left - groups <= 0;  // of this phase, for a chain
+    const int jq = w.j, ph = w.ph;
     w.next();
 
-    if (g_end == ng || w.done()) {
+    if (g_end == ng || range_ends) {
       // ---- the panel ends here (or the range does): emit the 16 columns this warp owns
       const int covered = g_end - g_begin;
       if constexpr (G != kGroup) {
@@ -524,6 +710,46 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
             acc1[mt][j] = 0.0f;
           }
       }
+      // What follows the sums: fixed per instantiation for a list, a property of the step in a chain.
+      int epi = EPI;
+      float r_even = 1.0f, r_odd = 1.0f;  // chain: row factors of tokens 2t and 2t + 1 (a folded rms-norm)
+      if constexpr (CHAIN) {
+        epi = q.epi;
+        if (q.rms_eps >= 0.0f) {
+          const int slot = jq & (kChainRmsSlots - 1);
+          const long long t0 = clock64();
+          while (rms_step[slot] != jq) {
+            if (clock64() - t0 > p.wait_limit) {
+              if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
+              return;
+            }
+          }
+          __threadfence_block();
+          r_even = rms_val[slot * 8 + 2 * t];
+          r_odd = rms_val[slot * 8 + 2 * t + 1];
+        }
+      }
+      auto addend = [&](int m, size_t n) -> float {
+        if constexpr (CHAIN) return __half2float(__ldcg(q.add + (size_t)m * q.add_stride + n));  // L2: other SMs wrote it
+        else return __half2float(p.add[(size_t)m * p.add_stride + n]);
+      };
+      // one finished output (and, for SwiGLU, its partner 8 columns on): the epilogue and the store
+      auto emit = [&](int m, size_t n, float v, float v_up, int j) {
+        if (CHAIN) {
+          const float r = (j & 1) ? r_odd : r_even;
+          v *= r;
+          v_up *= r;
+        }
+        if (epi == 2) {
+          // columns gid (gate) and gid + 8 (up) of the tile sit in the same lane: the tile's eight
+          // outputs silu(gate) * up go to columns 8 * tile + gid of y[M, N / 2]
+          if (j < 2) q.y[(size_t)m * (q.N >> 1) + (n - gid) / 2 + gid] = __float2half_rn(swiglu(v, v_up));
+        } else {
+          if (epi == 1) v += addend(m, n);
+          q.y[(size_t)m * q.N + n] = __float2half_rn(v);
+        }
+      };
+      bool final_here = false;  // chain: this CTA made the panel final
       const size_t n_lo = (size_t)(panel * kPanelTiles + warp) * kTileN + gid;
       if (covered == ng) {
         if (warp < R) {
@@ -532,30 +758,28 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int m = 8 * mt + 2 * t + (j & 1);
-              const size_t n = n_lo + (j >> 1) * 8;
-              if constexpr (EPI == 2) {
-                // columns gid (gate) and gid + 8 (up) of the tile sit in the same lane: the tile's
-                // eight outputs silu(gate) * up go to columns 8 * tile + gid of y[M, N / 2]
-                if (j < 2 && m < M)
-                  q.y[(size_t)m * (q.N >> 1) + (n_lo - gid) / 2 + gid] = __float2half_rn(swiglu(acc[mt][j], acc[mt][j + 2]));
-              } else if (m < M) {
-                const size_t at = (size_t)m * q.N + n;
-                float v = acc[mt][j];
-                if constexpr (EPI == 1) v += __half2float(p.add[(size_t)m * p.add_stride + n]);
-                q.y[at] = __float2half_rn(v);
-              }
+              if (m < M) emit(m, n_lo + (j >> 1) * 8, acc[mt][j], acc[mt][(j + 2) & 3], j);
             }
           }
         }
+        final_here = true;
       } else {
         // the panel is shared with neighbouring CTAs: its scratch slot is named after the first
         // range boundary that falls inside the panel (after the panel itself when every panel
         // has its own CTAs)
+        int unit = 0, total = 0;
+        if constexpr (CHAIN) {
+          unit = p.phase[ph].unit;
+          total = p.phase[ph].chunks;
+        } else {
+          unit = p.unit;
+          total = p.total_chunks;
+        }
         int k = panel;
-        if (p.unit > 0) {
+        if (unit > 0) {
           const long long ps = (long long)q.chunk_begin + (long long)panel * ng;
-          k = (int)(ps * gridDim.x / p.total_chunks);
-          while ((long long)p.total_chunks * k / gridDim.x <= ps) ++k;
+          k = (int)(ps * gridDim.x / total);
+          while ((long long)total * k / gridDim.x <= ps) ++k;
         }
         float* slot = reinterpret_cast<float*>(p.ws + (size_t)k * kSlotBytes);
         unsigned int* cnt = reinterpret_cast<unsigned int*>(slot + kSlotFloats);
@@ -585,26 +809,28 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
                 const int m = 8 * mt + 2 * t + (j & 1);
-                const size_t n = n_lo + (j >> 1) * 8;
                 if (m < M) {
                   float* a = slot + c_lo + (j >> 1) * 8 * kWsPad + m;
-                  const size_t at = (size_t)m * q.N + n;
-                  float v = __ldcg(a);
-                  if constexpr (EPI == 2) {
-                    // the up half (j >= 2) is read by the iteration of its gate and cleared by its own
-                    if (j < 2)
-                      q.y[(size_t)m * (q.N >> 1) + (n_lo - gid) / 2 + gid] =
-                          __float2half_rn(swiglu(v, __ldcg(a + 8 * kWsPad)));
-                  } else {
-                    if constexpr (EPI == 1) v += __half2float(p.add[(size_t)m * p.add_stride + n]);
-                    q.y[at] = __float2half_rn(v);
-                  }
+                  // SwiGLU: the up half (j >= 2) is read by the iteration of its gate and cleared by its own
+                  const float v = __ldcg(a);
+                  const float v_up = (epi == 2 && j < 2) ? __ldcg(a + 8 * kWsPad) : 0.0f;
+                  emit(m, n_lo + (j >> 1) * 8, v, v_up, j);
                   __stcg(a, 0.0f);
                 }
               }
             }
           }
           if (tid == 0) *cnt = 0;
+          final_here = true;
+        }
+      }
+      if constexpr (CHAIN) {
+        // A panel that is final counts towards the next phase's target: its outputs (and the cleared
+        // slot) are made visible, then one thread adds to the counter with release semantics.
+        if (final_here) {
+          __threadfence();
+          ptx::named_bar_sync(1, kConsumerThreads);
+          if (tid == 0) ptx::red_release_gpu(p.sync, 1u);
         }
       }
 #pragma unroll
@@ -612,6 +838,22 @@ gemv_decode_kernel(const __grid_constant__ DecodeParams<NB> p) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[mt][j] = 0.0f;
       g_begin = (g_end == ng) ? 0 : g_end;
+      if constexpr (CHAIN) {
+        if (range_ends && !w.done()) g_begin = w.g;  // the range of the next phase starts mid-panel, too
+      }
+    }
+  }
+  if constexpr (CHAIN) {
+    // The last CTA to finish leaves the two counters zero for the next launch.  The fence orders this
+    // CTA's additions to the panel counter before its arrival here.
+    if (tid == 0) {
+      __threadfence();
+      const unsigned prev = atomicAdd(p.sync + 1, 1u);
+      if (prev == gridDim.x - 1) {
+        __threadfence();
+        p.sync[0] = 0u;
+        p.sync[1] = 0u;
+      }
     }
   }
 }
@@ -650,7 +892,7 @@ cudaError_t launch_one(const DecodeParams<NB>& p, int grid, size_t smem, cudaStr
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(gemv_decode_kernel<MT, NB, ROT, EPI, G>,
+    cudaError_t e = cudaFuncSetAttribute(gemv_decode_kernel<MT, DecodeParams<NB>, ROT, EPI, G>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          // groups of 32 with more than 11 tokens need 117 KB for two stages
                                          (G == kGroup ? 112 : 120) * 1024);
@@ -667,7 +909,7 @@ cudaError_t launch_one(const DecodeParams<NB>& p, int grid, size_t smem, cudaStr
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemv_decode_kernel<MT, NB, ROT, EPI, G>, p);
+  return cudaLaunchKernelEx(&cfg, gemv_decode_kernel<MT, DecodeParams<NB>, ROT, EPI, G>, p);
 }
 
 template <int NB, int G = kGroup>
@@ -809,6 +1051,150 @@ cudaError_t launch_gemv_decode(const __half* x, const uint32_t* packed, const ui
     const int64_t stride = add_stride >= 0 ? add_stride : N;
     DecodeProblem q{x + m0 * K, packed, scales, y + m0 * (swiglu ? N / 2 : N), K, N, add ? add + m0 * stride : nullptr, swiglu, stride};
     const cudaError_t e = launch_batch_group<1>(&q, 1, Mc, workspace, stream, group);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------- a chain of dependent steps
+namespace {
+
+constexpr size_t kChainSmemExtra = 320;  // row factors of kChainRmsSlots steps and their tags
+
+template <bool ROT, int G>
+cudaError_t chain_kernel_setup(int* blocks_per_sm, size_t smem) {
+  auto kernel = gemv_decode_kernel<1, ChainParams, ROT, 0, G>;
+  static bool configured[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, kernel, kThreads, smem);
+}
+
+template <bool ROT, int G>
+cudaError_t chain_kernel_launch(const ChainParams& p, int grid, size_t smem, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemv_decode_kernel<1, ChainParams, ROT, 0, G>, p);
+}
+
+// One launch of at most kMaxChain steps.  Every CTA of the grid takes part in every phase, and a
+// phase waits for CTAs of the one before, so the whole grid has to be resident at once: the grid is
+// what the occupancy calculation says fits (two CTAs per SM).
+template <int G>
+cudaError_t launch_chain(const ChainStep* steps, int count, int M, void* workspace, cudaStream_t stream) {
+  const int sms = sm_count();
+  unsigned int* status = device_status_word();
+  if (!status) return cudaErrorUnknown;
+  static ChainParams p;  // 14 KB: too large for the stack of a small thread; guarded by the mutex below
+  static std::mutex lock;
+  std::lock_guard<std::mutex> guard(lock);
+  p.ws = static_cast<uint8_t*>(workspace);
+  p.status = status;
+  p.sync = reinterpret_cast<unsigned int*>(p.ws + (size_t)kMaxSlots * kSlotBytes);
+  p.M = M;
+  p.count = count;
+  p.wait_limit = wait_limit_cycles();
+  p.skip_copies = tune(kTuneSkipCopies) == 1;
+  p.xsum_offset = x_offset(G) + M * kXRowBytes;
+  p.stage_bytes = (p.xsum_offset + kStageGroups * 32 * (int)sizeof(float) + 127) & ~127;
+  int stages = kRingBudget / p.stage_bytes;
+  stages = stages > kMaxStages ? kMaxStages : (stages < 2 ? 2 : stages);
+  p.stages = stages;
+  const size_t smem =
+      128 + (size_t)stages * p.stage_bytes + 3 * kMaxStages * sizeof(uint64_t) + 16 + 64 + kChainSmemExtra;
+  const bool rot = M >= 5;
+  int per_sm = 0;
+  cudaError_t e = rot ? chain_kernel_setup<true, G>(&per_sm, smem) : chain_kernel_setup<false, G>(&per_sm, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  if (per_sm > 2) per_sm = 2;
+  int grid = per_sm * sms;
+  if (grid > kMaxSlots - 1) grid = kMaxSlots - 1;
+
+  int phases = 0;
+  unsigned int panels_before = 0;
+  for (int j = 0; j < count; ++j) {
+    const ChainStep& st = steps[j];
+    if (j == 0 || st.after_previous) {
+      ChainPhase& f = p.phase[phases];
+      f.first = j;
+      f.chunks = 0;
+      f.wait_target = panels_before;
+      ++phases;
+    }
+    ChainPhase& f = p.phase[phases - 1];
+    ChainProb& q = p.prob[j];
+    q.x = st.x;
+    q.packed = reinterpret_cast<const uint8_t*>(st.packed);
+    q.scales = reinterpret_cast<const uint8_t*>(st.scales);
+    q.y = st.y;
+    q.add = st.add;
+    q.add_stride = st.add_stride;
+    q.K = (int)st.K;
+    q.N = (int)st.N;
+    q.ng = (int)(st.K / kGroup);
+    q.nbs = (int)(st.N / kTileN);
+    q.panels = (q.nbs + kPanelTiles - 1) / kPanelTiles;
+    q.chunk_begin = f.chunks;
+    q.epi = st.epi;
+    q.phase = phases - 1;
+    q.rms_eps = st.rms_eps;
+    if ((long long)f.chunks + (long long)q.panels * q.ng > 0x7FFFFFFFLL / 512) return cudaErrorInvalidValue;
+    f.chunks += q.panels * q.ng;
+    f.last = j + 1;
+    panels_before += (unsigned)q.panels;
+  }
+  p.phases = phases;
+  for (int i = 0; i < phases; ++i) {
+    ChainPhase& f = p.phase[i];
+    f.unit = 1;
+    if (f.last - f.first == 1) {
+      // a lone step is cut as a lone problem is: whole panels when that loads the CTAs evenly,
+      // else a fixed number of CTAs per panel, each with a slice of the panel's groups
+      const ChainProb& q = p.prob[f.first];
+      const int per = (q.panels + grid - 1) / grid;
+      if (q.panels >= grid && (double)q.panels / ((double)per * grid) >= 0.97) f.unit = q.ng;
+      if (q.panels < grid) {
+        int slices = grid / q.panels < q.ng ? grid / q.panels : q.ng;
+        if (slices == 2 && q.ng <= 16) slices = 1;
+        f.unit = -slices;
+      }
+      // tl_e0m4_tuning_set("decode_split" / "decode_slices") force the cut, as for a lone problem
+      if (tune(kTuneDecodeSplit) == 1) f.unit = q.ng;
+      if (tune(kTuneDecodeSplit) == 2) f.unit = 1;
+      const int64_t forced = tune(kTuneDecodeSlices);
+      if (forced >= 1 && forced <= q.ng && forced * q.panels <= grid) f.unit = -(int)forced;
+    }
+  }
+  e = rot ? chain_kernel_launch<true, G>(p, grid, smem, stream) : chain_kernel_launch<false, G>(p, grid, smem, stream);
+  count_launch();
+  return e;
+}
+
+}  // namespace
+
+size_t decode_chain_workspace_bytes() { return (size_t)kMaxSlots * kSlotBytes + 256; }
+
+cudaError_t launch_gemv_decode_chain(const ChainStep* steps, int count, int M, void* workspace, cudaStream_t stream,
+                                     int group) {
+  for (int j0 = 0; j0 < count; j0 += kMaxChain) {
+    const int n = count - j0 < kMaxChain ? count - j0 : kMaxChain;
+    const cudaError_t e = group == 32   ? launch_chain<32>(steps + j0, n, M, workspace, stream)
+                          : group == 64 ? launch_chain<64>(steps + j0, n, M, workspace, stream)
+                                        : launch_chain<kGroup>(steps + j0, n, M, workspace, stream);
     if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();

@@ -141,3 +141,22 @@ def test_e0m8_sizes_and_argument_errors(lib):
     assert L.tl_e0m8_matmul_batch(ptr, 1, 1, 128, a, 16, None) == 5  # TL_ERR_WORKSPACE
     assert lib.tl_e0m4_launch_count() == before
     assert lib.tl_e0m8_matmul_workspace(1, 100, 16) == 0
+
+
+def test_chain_argument_errors_come_back_before_any_launch(lib):
+    L = lib.lib()
+    a = 0x10000
+    st = lib.Step(a, a, a, a, None, 128, 16, 0, 0, 0, 0.0)
+    ptr = lambda s: ctypes.cast(ctypes.pointer(s), ctypes.c_void_p)
+    big = 1 << 30
+    before = lib.tl_e0m4_launch_count()
+    assert L.tl_e0m4_matmul_chain(None, 1, 1, 128, a, big, None) == 1
+    assert L.tl_e0m4_matmul_chain(ptr(st), 0, 1, 128, a, big, None) == 2
+    assert L.tl_e0m4_matmul_chain(ptr(st), 1, 9, 128, a, big, None) == 2       # more than 8 tokens
+    assert L.tl_e0m4_matmul_chain(ptr(st), 1, 1, 128, a, 16, None) == 5        # workspace too small
+    assert L.tl_e0m4_matmul_chain(ptr(lib.Step(a, a, a, a, None, 128, 16, 1, 0, 0, 0.0)), 1, 1, 128, a, big, None) == 1
+    assert L.tl_e0m4_matmul_chain(ptr(lib.Step(a, a, a, a, a + 2, 128, 16, 2, 0, 0, 0.0)), 1, 1, 128, a, big, None) == 3
+    assert L.tl_e0m4_matmul_chain(ptr(lib.Step(a, a, a, a, None, 128, 16, 7, 0, 0, 0.0)), 1, 1, 128, a, big, None) == 2
+    assert L.tl_e0m4_matmul_chain(ptr(lib.Step(a, a, a, a, None, 100, 16, 0, 0, 0, 0.0)), 1, 1, 128, a, big, None) == 2
+    assert L.tl_e0m4_matmul_chain(ptr(lib.Step(a, a, a, a, None, 128, 16, 0, 0, 1, -1.0)), 1, 1, 128, a, big, None) == 2
+    assert lib.tl_e0m4_launch_count() == before
