@@ -35,6 +35,14 @@
 #include "tuning.h"
 
 namespace tl {
+#ifdef TL_CHAIN_TRACE
+__device__ unsigned long long g_trace[8][256];
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define TRACE(k, j) do { if (blockIdx.x == TRACE_CTA && (j) < 256) g_trace[k][j] = gtime(); } while (0)
+#define TRACE_CTA 0
+#else
+#define TRACE(k, j) do {} while (0)
+#endif
 namespace {
 
 constexpr int kConsumerWarps = kPanelTiles;          // one warp per column block of a panel
@@ -151,9 +159,14 @@ __device__ __forceinline__ void cta_range(int total, int unit, int ng, int panel
     c0 = panel * ng + ng * i / s;
     c1 = panel * ng + ng * (i + 1) / s;
   } else {
-    const long long units = total / unit;
-    c0 = (int)(units * blockIdx.x / gridDim.x) * unit;
-    c1 = (int)(units * (blockIdx.x + 1) / gridDim.x) * unit;
+    const unsigned int units = (unsigned int)(total / unit), b = blockIdx.x, n = gridDim.x;
+    if (units < 0xFFFFFFFFu / (n + 1)) {  // the products fit 32 bits: a 64-bit division costs hundreds of cycles
+      c0 = (int)(units * b / n) * unit;
+      c1 = (int)(units * (b + 1) / n) * unit;
+    } else {
+      c0 = (int)((unsigned long long)units * b / n) * unit;
+      c1 = (int)((unsigned long long)units * (b + 1) / n) * unit;
+    }
   }
 }
 
@@ -392,10 +405,11 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           const unsigned int target = p.phase[wx.ph].wait_target;
           if (seen < target) {
             seen = ptx::ld_acquire_gpu(p.sync);
-            if (seen >= target) ptx::fence_proxy_async_all();
+            if (seen >= target) { TRACE(3, wx.j); ptx::fence_proxy_async_all(); }
           }
           if (seen >= target) {
             issue_x(wx, sx);
+            TRACE(4, wx.j);
             wx.next();
             ++ix;
             if (++sx == S) sx = 0;
@@ -455,6 +469,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
         if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
         return;
       }
+      if (lane == 0) TRACE(5, w.j);
       const uint32_t st = ring_h + s * p.stage_bytes;
       float* xsum = reinterpret_cast<float*>(ring + (size_t)s * p.stage_bytes + p.xsum_offset);
       const bool live = sub < w.groups();
@@ -505,14 +520,23 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
             for (int m = 0; m < M; ++m) {
               const uint4* row = reinterpret_cast<const uint4*>(q.x + (size_t)m * q.K);
               float ss = 0.0f;
-              for (int i = lane; i < q.K / 8; i += 32) {
-                const uint4 v = __ldcg(row + i);
-                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
-                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
-                const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&v.z));
-                const float2 f3 = __half22float2(*reinterpret_cast<const __half2*>(&v.w));
-                ss += (f0.x * f0.x + f0.y * f0.y) + (f1.x * f1.x + f1.y * f1.y) + (f2.x * f2.x + f2.y * f2.y) +
-                      (f3.x * f3.x + f3.y * f3.y);
+              const int vecs = q.K / 8;  // a multiple of 16
+              for (int i0 = 0; i0 < vecs; i0 += 8 * 32) {
+                uint4 v[8];  // eight loads in flight per lane: the row costs one or two round trips to L2
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                  const int i = i0 + u * 32 + lane;
+                  v[u] = i < vecs ? __ldcg(row + i) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                  const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&v[u].x));
+                  const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&v[u].y));
+                  const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&v[u].z));
+                  const float2 f3 = __half22float2(*reinterpret_cast<const __half2*>(&v[u].w));
+                  ss += (f0.x * f0.x + f0.y * f0.y) + (f1.x * f1.x + f1.y * f1.y) + (f2.x * f2.x + f2.y * f2.y) +
+                        (f3.x * f3.x + f3.y * f3.y);
+                }
               }
 #pragma unroll
               for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, off);
@@ -576,6 +600,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
       if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
       return;  // every wait in this kernel is bounded, so the other warps leave as well
     }
+    if (tid == 0) TRACE(0, w.j);
     if (warp < R) {
       const uint32_t st = ring_u32 + s * p.stage_bytes;
       const uint32_t wt_base = st + warp * kTileBytes + lane * 16;
@@ -696,9 +721,9 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
     const int g_end = w.g + groups;
     const bool range_ends = w.left - groups <= 0;  // of this phase, for a chain
     const int jq = w.j, ph = w.ph;
-    w.next();
 
     if (g_end == ng || range_ends) {
+      if (tid == 0) TRACE(1, jq);
       // ---- the panel ends here (or the range does): emit the 16 columns this warp owns
       const int covered = g_end - g_begin;
       if constexpr (G != kGroup) {
@@ -825,12 +850,12 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
         }
       }
       if constexpr (CHAIN) {
-        // A panel that is final counts towards the next phase's target: its outputs (and the cleared
-        // slot) are made visible, then one thread adds to the counter with release semantics.
+        // A panel that is final counts towards the next phase's target.  The barrier orders every
+        // consumer's stores (outputs, cleared slot) before thread 0, whose addition to the counter
+        // has release semantics at GPU scope, which is cumulative over what the barrier ordered.
         if (final_here) {
-          __threadfence();
           ptx::named_bar_sync(1, kConsumerThreads);
-          if (tid == 0) ptx::red_release_gpu(p.sync, 1u);
+          if (tid == 0) { TRACE(6, jq); ptx::red_release_gpu(p.sync, 1u); TRACE(2, jq); }
         }
       }
 #pragma unroll
@@ -838,9 +863,12 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[mt][j] = 0.0f;
       g_begin = (g_end == ng) ? 0 : g_end;
-      if constexpr (CHAIN) {
-        if (range_ends && !w.done()) g_begin = w.g;  // the range of the next phase starts mid-panel, too
-      }
+    }
+    // (a chain's walk may have to find the CTA's range of the next phase here: after the panel has
+    // been published, not before)
+    w.next();
+    if constexpr (CHAIN) {
+      if (range_ends && !w.done()) g_begin = w.g;  // the range of the next phase may start mid-panel
     }
   }
   if constexpr (CHAIN) {
@@ -1186,6 +1214,9 @@ cudaError_t launch_chain(const ChainStep* steps, int count, int M, void* workspa
 
 }  // namespace
 
+#ifdef TL_CHAIN_TRACE
+extern "C" void tl_debug_trace(unsigned long long* out) { cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * 8 * 256); }
+#endif
 size_t decode_chain_workspace_bytes() { return (size_t)kMaxSlots * kSlotBytes + 256; }
 
 cudaError_t launch_gemv_decode_chain(const ChainStep* steps, int count, int M, void* workspace, cudaStream_t stream,
