@@ -382,7 +382,8 @@ uint64_t tl_e0m4_launch_count(void);
  * fewest token tiles), "list_pair" (0 / 1), "batch_tc_min" (first token count of a list that takes
  * the tensor-core kernel), "register_max_m" (most tokens of a single call on the register kernel,
  * 1..16), "decode_split" (1 whole panels per CTA, 2 stream-K ranges), "decode_slices" (CTAs per
- * panel), "decode_ctas_per_sm" (1, 2), "decode_rot_min", "wait_limit_cycles" (SM cycles after
+ * panel), "decode_ctas_per_sm" (1, 2), "decode_rot_min", "decode_cluster" (0: CTAs that share a panel add
+ * their sums up in the global scratch instead of a cluster's shared memory), "wait_limit_cycles" (SM cycles after
  * which a device-side wait gives up and raises TL_ERR_TIMEOUT in the status word; about two seconds
  * by default), "skip_copies" (1: the producers of the matmul kernels issue no copies, so that with
  * a short wait limit every wait runs out while nothing is in flight: the safe way to see the

@@ -587,7 +587,7 @@ uint64_t tl_e0m4_launch_count(void) { return g_launches.load(std::memory_order_r
 tl_status tl_e0m4_tuning_set(const char* key, int64_t value) {
   static const char* const names[kTuneCount] = {
       "ksplit", "tc_pair", "tc_big", "tc_mtiles", "list_pair", "batch_tc_min", "decode_split", "decode_slices",
-      "decode_ctas_per_sm", "decode_rot_min", "wait_limit_cycles", "skip_copies", "register_max_m"};
+      "decode_ctas_per_sm", "decode_rot_min", "wait_limit_cycles", "skip_copies", "register_max_m", "decode_cluster"};
   if (!key) {
     for (auto& v : g_tuning) v.store(-1, std::memory_order_relaxed);
     return TL_OK;

@@ -35,14 +35,6 @@
 #include "tuning.h"
 
 namespace tl {
-#ifdef TL_CHAIN_TRACE
-__device__ unsigned long long g_trace[8][256];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define TRACE(k, j) do { if (blockIdx.x == TRACE_CTA && (j) < 256) g_trace[k][j] = gtime(); } while (0)
-#define TRACE_CTA 0
-#else
-#define TRACE(k, j) do {} while (0)
-#endif
 namespace {
 
 constexpr int kConsumerWarps = kPanelTiles;          // one warp per column block of a panel
@@ -62,6 +54,16 @@ constexpr int kXRowBytes = kStageGroups * 256 + 32;
 constexpr int kWsPad = 16;                           // scratch floats per output column
 constexpr int kMaxStages = 4;
 
+// Panels whose k groups are shared by the s = 2, 4 or 8 CTAs of (a part of) a cluster meet in
+// shared memory instead of the global scratch: every CTA sends the partial sums of tile t to the
+// CTA with rank t % s of its group, which adds the s contributions of its 8 / s tiles and stores
+// them.  The receiving buffer: [sender x tile: 8][16 columns][8 MT tokens] fp32, and one barrier.
+__host__ __device__ constexpr int red_bytes(int mt) { return kPanelTiles * kTileN * 8 * mt * 4; }  // 8 tokens per block of tokens
+constexpr int kRedOffset = (3 * kMaxStages + 48) * 8;  // from the barriers: past flags, zero block and row factors
+constexpr int kSmemTail = 3 * kMaxStages * 8 + 16 + 64;             // barriers, flags, zero block
+// ... row factors, exchange barrier and buffer
+__host__ __device__ constexpr int smem_tail_cluster(int mt) { return kRedOffset + 16 + red_bytes(mt); }
+
 constexpr int kSlotFloats = kPanelTiles * kTileN * kWsPad;  // fp32 partial sums of one panel
 constexpr int kSlotBytes = kSlotFloats * 4 + 128;           // + the panel's chunk counter
 constexpr int kMaxSlots = 320;                              // >= number of CTAs of a launch
@@ -80,6 +82,7 @@ struct Prob {
 template <int NB>
 struct DecodeParams {
   static constexpr bool kChain = false;
+  static constexpr bool kCluster = NB == 1;  // lone problems may be launched as clusters (see red_bytes)
   uint8_t* ws;            // kMaxSlots slots of {fp32 [128][16] partial sums, chunk counter}, zero between calls
   unsigned int* status;   // device status word (0 = fine)
   int M;
@@ -95,6 +98,7 @@ struct DecodeParams {
   long long add_stride;   // elements between the addend's token rows: N, or 0 for a bias row shared by all tokens
   long long wait_limit;   // SM cycles after which a bounded wait gives up
   int skip_copies;        // diagnostics: the producer issues nothing, so every wait runs out
+  int cluster;            // CTAs per thread-block cluster of this launch (1 = no clusters)
 };
 
 // ---- a chain of steps that may depend on one another (tl_e0m4_matmul_chain)
@@ -122,7 +126,7 @@ struct ChainPhase {
   int first, last;        // steps [first, last) of the launch
   int chunks;             // chunks of the phase
   int unit;               // as DecodeParams::unit, for this phase
-  unsigned int wait_target;  // panels of all earlier phases: the phase's activations exist once that many are final
+  unsigned int wait_target;  // 8 x the panels of all earlier phases: the phase's activations exist once that much is final
 };
 
 constexpr int kMaxChain = 128;       // steps per launch (their descriptors travel as kernel parameters)
@@ -130,9 +134,10 @@ constexpr int kChainRmsSlots = 8;    // row factors are kept for this many steps
 
 struct ChainParams {
   static constexpr bool kChain = true;
+  static constexpr bool kCluster = true;
   uint8_t* ws;            // the scratch slots of DecodeParams::ws
   unsigned int* status;
-  unsigned int* sync;     // [0] panels made final so far in this launch, [1] CTAs that have finished; zero between launches
+  unsigned int* sync;     // [0] eighths of panels made final so far in this launch, [1] CTAs that have finished; zero between launches
   int M;
   int count;
   int phases;
@@ -141,6 +146,7 @@ struct ChainParams {
   int xsum_offset;
   long long wait_limit;
   int skip_copies;
+  int cluster;            // CTAs per thread-block cluster of this launch (1 = no clusters)
   ChainProb prob[kMaxChain];
   ChainPhase phase[kMaxChain];
 };
@@ -308,6 +314,8 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
   // chain: row factors of the last kChainRmsSlots steps, [slot][8 tokens], and the step each slot holds
   float* rms_val = reinterpret_cast<float*>(bars + 3 * kMaxStages + 10);
   volatile int* rms_step = reinterpret_cast<volatile int*>(rms_val + kChainRmsSlots * 8);
+  const uint32_t red_bar = ptx::smem_u32(bars) + kRedOffset;   // cluster launches: the exchange barrier ...
+  const uint32_t red_buf = red_bar + 16;                       // ... and the buffer the group's CTAs write into
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -324,11 +332,18 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
       ptx::mbar_init(xbar0 + 8 * s, 1);
     }
     flags[0] = 0;
+    if constexpr (PT::kCluster) {
+      if (p.cluster > 1) ptx::mbar_init(red_bar, kConsumerWarps);
+    }
     ptx::fence_mbar_init();
   }
   if (tid < 16) reinterpret_cast<uint32_t*>(bars + 3 * kMaxStages + 2)[tid] = 0u;
   if (CHAIN && tid < kChainRmsSlots) rms_step[tid] = -1;
   __syncthreads();
+  if constexpr (PT::kCluster) {
+    // every CTA's exchange barrier exists before a neighbour arrives on it (all threads are still here)
+    if (p.cluster > 1) ptx::cluster_sync_all();
+  }
   ptx::pdl_launch_dependents();
 
   // this CTA's contiguous range of chunks (a chain has one per phase: see StageWalk)
@@ -405,11 +420,10 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           const unsigned int target = p.phase[wx.ph].wait_target;
           if (seen < target) {
             seen = ptx::ld_acquire_gpu(p.sync);
-            if (seen >= target) { TRACE(3, wx.j); ptx::fence_proxy_async_all(); }
+            if (seen >= target) ptx::fence_proxy_async_all();
           }
           if (seen >= target) {
             issue_x(wx, sx);
-            TRACE(4, wx.j);
             wx.next();
             ++ix;
             if (++sx == S) sx = 0;
@@ -469,7 +483,6 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
         if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
         return;
       }
-      if (lane == 0) TRACE(5, w.j);
       const uint32_t st = ring_h + s * p.stage_bytes;
       float* xsum = reinterpret_cast<float*>(ring + (size_t)s * p.stage_bytes + p.xsum_offset);
       const bool live = sub < w.groups();
@@ -589,6 +602,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
   const uint32_t ring_u32 = ptx::smem_u32(ring);
 
   StageWalk<PT> w = make_walk();
+  [[maybe_unused]] uint32_t red_phase = 0;  // cluster launches: parity of the next exchange
   int g_begin = w.g;
   int s = 0, phase = 0;
   while (!w.done()) {
@@ -600,7 +614,6 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
       if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
       return;  // every wait in this kernel is bounded, so the other warps leave as well
     }
-    if (tid == 0) TRACE(0, w.j);
     if (warp < R) {
       const uint32_t st = ring_u32 + s * p.stage_bytes;
       const uint32_t wt_base = st + warp * kTileBytes + lane * 16;
@@ -723,7 +736,6 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
     const int jq = w.j, ph = w.ph;
 
     if (g_end == ng || range_ends) {
-      if (tid == 0) TRACE(1, jq);
       // ---- the panel ends here (or the range does): emit the 16 columns this warp owns
       const int covered = g_end - g_begin;
       if constexpr (G != kGroup) {
@@ -774,7 +786,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           q.y[(size_t)m * q.N + n] = __float2half_rn(v);
         }
       };
-      bool final_here = false;  // chain: this CTA made the panel final
+      int final_share = 0;  // chain: eighths of the panel that this CTA made final (8 = the whole panel)
       const size_t n_lo = (size_t)(panel * kPanelTiles + warp) * kTileN + gid;
       if (covered == ng) {
         if (warp < R) {
@@ -787,7 +799,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
             }
           }
         }
-        final_here = true;
+        final_share = kPanelTiles;
       } else {
         // the panel is shared with neighbouring CTAs: its scratch slot is named after the first
         // range boundary that falls inside the panel (after the panel itself when every panel
@@ -800,7 +812,75 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           unit = p.unit;
           total = p.total_chunks;
         }
+        bool exchanged = false;
+        if constexpr (PT::kCluster) {
+          if (unit < 0 && p.cluster > 1) {
+            // ---- the s CTAs that share this panel are neighbours in a cluster: exchange through shared memory
+            exchanged = true;
+            const int s_grp = -unit;
+            const int my_i = (int)(blockIdx.x % (unsigned)s_grp);               // slice of the panel = rank in the group
+            const uint32_t base = ptx::cluster_ctarank() - (uint32_t)my_i;     // cluster rank of the group's first CTA
+            const uint32_t dst = base + (uint32_t)(warp % s_grp);              // who finishes this warp's tile
+            const int per = kPanelTiles / s_grp;                               // tiles every CTA finishes
+            if (warp < R) {
+              constexpr int kRedPad = 8 * MT;
+              const uint32_t to = ptx::mapa(red_buf + (uint32_t)((my_i * per + warp / s_grp) * kTileN * kRedPad * 4), dst);
+#pragma unroll
+              for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int m = 8 * mt + 2 * t + (j & 1);
+                  if (m < M) ptx::st_cluster_f32(to + (uint32_t)(((gid + (j >> 1) * 8) * kRedPad + m) * 4), acc[mt][j]);
+                }
+              }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_release_cluster(ptx::mapa(red_bar, dst));
+            // all eight warps of all s CTAs have arrived here once the phase completes
+            if (!ptx::mbar_wait_bounded_cluster(red_bar, red_phase, p.wait_limit)) {
+              if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
+              return;
+            }
+            red_phase ^= 1;
+            const int tile = warp * s_grp + my_i;  // the tile this warp finishes, if it has one
+            if (warp < per && tile < R) {
+              const size_t n_out = (size_t)(panel * kPanelTiles + tile) * kTileN + gid;
+              // the s contributions to this lane's four sums: all loads first, then the additions
+              const uint32_t mine = red_buf + (uint32_t)(((warp * kTileN + gid) * (8 * MT) + 2 * t) * 4);
+              const uint32_t src_stride = (uint32_t)(per * kTileN * 8 * MT * 4);
+#pragma unroll
+              for (int mt = 0; mt < MT; ++mt) {
+                float2 part[kPanelTiles][2];  // [sender][column gid, column gid + 8]: tokens 2t and 2t + 1
+#pragma unroll
+                for (int src = 0; src < kPanelTiles; ++src) {
+                  part[src][0] = part[src][1] = make_float2(0.0f, 0.0f);
+                  if (src < s_grp) {
+                    part[src][0] = ptx::lds64f(mine + src * src_stride + mt * 32);
+                    part[src][1] = ptx::lds64f(mine + src * src_stride + mt * 32 + 8 * (8 * MT) * 4);
+                  }
+                }
+                float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                for (int src = 0; src < kPanelTiles; ++src) {
+                  v[0] += part[src][0].x;
+                  v[1] += part[src][0].y;
+                  v[2] += part[src][1].x;
+                  v[3] += part[src][1].y;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int m = 8 * mt + 2 * t + (j & 1);
+                  if (m < M) emit(m, n_out + (j >> 1) * 8, v[j], v[(j + 2) & 3], j);
+                }
+              }
+            }
+            final_share = kPanelTiles / s_grp;
+          }
+        }
         int k = panel;
+        if (exchanged) {
+          // done above
+        } else {
         if (unit > 0) {
           const long long ps = (long long)q.chunk_begin + (long long)panel * ng;
           k = (int)(ps * gridDim.x / total);
@@ -846,16 +926,17 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
             }
           }
           if (tid == 0) *cnt = 0;
-          final_here = true;
+          final_share = kPanelTiles;
         }
+        }  // !exchanged
       }
       if constexpr (CHAIN) {
         // A panel that is final counts towards the next phase's target.  The barrier orders every
         // consumer's stores (outputs, cleared slot) before thread 0, whose addition to the counter
         // has release semantics at GPU scope, which is cumulative over what the barrier ordered.
-        if (final_here) {
+        if (final_share > 0) {
           ptx::named_bar_sync(1, kConsumerThreads);
-          if (tid == 0) { TRACE(6, jq); ptx::red_release_gpu(p.sync, 1u); TRACE(2, jq); }
+          if (tid == 0) ptx::red_release_gpu(p.sync, (unsigned)final_share);
         }
       }
 #pragma unroll
@@ -916,14 +997,16 @@ constexpr int kRingBudget = 110 * 1024;
 
 template <int MT, int NB, bool ROT, int EPI, int G>
 cudaError_t launch_one(const DecodeParams<NB>& p, int grid, size_t smem, cudaStream_t stream) {
+  if (p.cluster > 1) smem += smem_tail_cluster(MT) - kSmemTail;  // the exchange buffer of a cluster launch
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64 || !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(gemv_decode_kernel<MT, DecodeParams<NB>, ROT, EPI, G>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         // groups of 32 with more than 11 tokens need 117 KB for two stages
-                                         (G == kGroup ? 112 : 120) * 1024);
+                                         // groups of 32 with more than 11 tokens need 117 KB for two stages;
+                                         // cluster launches add their exchange buffer
+                                         (G == kGroup ? 116 : 126) * 1024);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
@@ -932,12 +1015,52 @@ cudaError_t launch_one(const DecodeParams<NB>& p, int grid, size_t smem, cudaStr
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (p.cluster > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)p.cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   return cudaLaunchKernelEx(&cfg, gemv_decode_kernel<MT, DecodeParams<NB>, ROT, EPI, G>, p);
+}
+
+// How many clusters of `size` CTAs of the lone-problem kernel can be resident at once (0 if the
+// question cannot be answered).  All instantiations have the same block size and, for a given
+// shared-memory size, the same footprint, so one of them answers for all; cached per device.
+int lone_max_clusters(int size, size_t smem) {
+  static std::atomic<int> cache[64][4];
+  int dev = 0;
+  cudaGetDevice(&dev);
+  const int slot = size == 8 ? 3 : (size == 4 ? 2 : 1);
+  if (dev >= 0 && dev < 64) {
+    const int c = cache[dev][slot].load(std::memory_order_relaxed);
+    if (c != 0) return c > 0 ? c : 0;
+  }
+  auto kernel = gemv_decode_kernel<1, DecodeParams<1>, false, 0, kGroup>;
+  int clusters = 0;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024) == cudaSuccess) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(size * 64));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) != cudaSuccess) clusters = 0;
+  }
+  (void)cudaGetLastError();
+  if (dev >= 0 && dev < 64) cache[dev][slot].store(clusters > 0 ? clusters : -1, std::memory_order_relaxed);
+  return clusters;
 }
 
 template <int NB, int G = kGroup>
@@ -957,6 +1080,7 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
   p.add_stride = count == 1 && probs[0].add_stride >= 0 ? probs[0].add_stride : probs[0].N;
   p.wait_limit = wait_limit_cycles();
   p.skip_copies = tune(kTuneSkipCopies) == 1;
+  p.cluster = 1;
   long long total = 0;
   for (int j = 0; j < count; ++j) {
     Prob& q = p.prob[j];
@@ -1004,6 +1128,20 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
     }
     if (forced_slices > 0 && split_mode < 0) slices = (int)forced_slices;
     if (slices > 0 && slices <= p.prob[0].ng && (long long)panels * slices <= grid) {
+      // Two, four or eight CTAs per panel are launched as a cluster and add their partial sums up in
+      // shared memory, which costs a fraction of the round trips through the global scratch; other
+      // counts are rounded down to such a cluster (tl_e0m4_tuning_set("decode_cluster", 0) keeps them).
+      // (only where that keeps at least three quarters of the CTAs: seven slices stay seven).
+      if (NB == 1 && tune(kTuneDecodeCluster) != 0 && slices >= 2) {
+        const int pow2 = slices >= 8 ? 8 : (slices >= 4 ? 4 : 2);
+        // ... and where all the clusters can be resident at once: a second wave would cost more
+        // (asked for the largest shared-memory size a cluster launch uses: three stages at one token)
+        const bool fits = panels <= lone_max_clusters(pow2, 128 + 3 * 36480 + smem_tail_cluster(1));
+        if (fits && (pow2 * 4 >= slices * 3 || tune(kTuneDecodeCluster) == 1)) {
+          slices = pow2;
+          p.cluster = slices;
+        }
+      }
       p.unit = -slices;
       grid = panels * slices;
     }
@@ -1012,7 +1150,8 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
   const int mt = M <= 8 ? 1 : 2;
   p.xsum_offset = x_offset(G) + M * kXRowBytes;
   p.stage_bytes = (p.xsum_offset + kStageGroups * 32 * (int)sizeof(float) + 127) & ~127;
-  int stages = kRingBudget / p.stage_bytes;
+  // (a cluster launch gives the room of its exchange buffer back, so that two CTAs still fit an SM)
+  int stages = (kRingBudget - (p.cluster > 1 ? smem_tail_cluster(mt) - kSmemTail : 0)) / p.stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : (stages < 2 ? 2 : stages);
   p.stages = stages;
   const size_t smem = 128 + (size_t)stages * p.stage_bytes + 3 * kMaxStages * sizeof(uint64_t) + 16 + 64;
@@ -1087,8 +1226,6 @@ cudaError_t launch_gemv_decode(const __half* x, const uint32_t* packed, const ui
 // ------------------------------------------------------------- a chain of dependent steps
 namespace {
 
-constexpr size_t kChainSmemExtra = 320;  // row factors of kChainRmsSlots steps and their tags
-
 template <bool ROT, int G>
 cudaError_t chain_kernel_setup(int* blocks_per_sm, size_t smem) {
   auto kernel = gemv_decode_kernel<1, ChainParams, ROT, 0, G>;
@@ -1096,11 +1233,31 @@ cudaError_t chain_kernel_setup(int* blocks_per_sm, size_t smem) {
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 126 * 1024);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, kernel, kThreads, smem);
+}
+
+// How many clusters of `size` CTAs can be resident at once.
+template <bool ROT, int G>
+cudaError_t chain_max_clusters(int* clusters, size_t smem, int size) {
+  int unused = 0;
+  cudaError_t e = chain_kernel_setup<ROT, G>(&unused, smem);  // sets the shared-memory attribute
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(size * 64));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)size;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(clusters, gemv_decode_kernel<1, ChainParams, ROT, 0, G>, &cfg);
 }
 
 template <bool ROT, int G>
@@ -1110,11 +1267,18 @@ cudaError_t chain_kernel_launch(const ChainParams& p, int grid, size_t smem, cud
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (p.cluster > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)p.cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   return cudaLaunchKernelEx(&cfg, gemv_decode_kernel<1, ChainParams, ROT, 0, G>, p);
 }
 
@@ -1138,19 +1302,34 @@ cudaError_t launch_chain(const ChainStep* steps, int count, int M, void* workspa
   p.skip_copies = tune(kTuneSkipCopies) == 1;
   p.xsum_offset = x_offset(G) + M * kXRowBytes;
   p.stage_bytes = (p.xsum_offset + kStageGroups * 32 * (int)sizeof(float) + 127) & ~127;
-  int stages = kRingBudget / p.stage_bytes;
+  int stages = (kRingBudget - (smem_tail_cluster(1) - kSmemTail)) / p.stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : (stages < 2 ? 2 : stages);
   p.stages = stages;
-  const size_t smem =
-      128 + (size_t)stages * p.stage_bytes + 3 * kMaxStages * sizeof(uint64_t) + 16 + 64 + kChainSmemExtra;
+  const size_t smem = 128 + (size_t)stages * p.stage_bytes + smem_tail_cluster(1);
   const bool rot = M >= 5;
-  int per_sm = 0;
-  cudaError_t e = rot ? chain_kernel_setup<true, G>(&per_sm, smem) : chain_kernel_setup<false, G>(&per_sm, smem);
-  if (e != cudaSuccess) return e;
-  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  if (per_sm > 2) per_sm = 2;
-  int grid = per_sm * sms;
-  if (grid > kMaxSlots - 1) grid = kMaxSlots - 1;
+  // Clusters of eight neighbouring CTAs, so that the CTAs that share a panel can add their sums up
+  // in shared memory; the grid is what can be resident at once, in whole clusters.  Where clusters
+  // would leave more than a quarter of the SMs' room unused, the launch does without them.
+  int grid = 0;
+  p.cluster = 1;
+  if (tune(kTuneDecodeCluster) != 0) {
+    int clusters = 0;
+    const cudaError_t ce = rot ? chain_max_clusters<true, G>(&clusters, smem, 8) : chain_max_clusters<false, G>(&clusters, smem, 8);
+    if (ce == cudaSuccess && clusters * 8 * 4 >= 2 * sms * 3) {
+      p.cluster = 8;
+      grid = clusters * 8 < 2 * sms / 8 * 8 ? clusters * 8 : 2 * sms / 8 * 8;
+    }
+    (void)cudaGetLastError();
+  }
+  if (p.cluster == 1) {
+    int per_sm = 0;
+    const cudaError_t e = rot ? chain_kernel_setup<true, G>(&per_sm, smem) : chain_kernel_setup<false, G>(&per_sm, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+    if (per_sm > 2) per_sm = 2;
+    grid = per_sm * sms;
+  }
+  if (grid > kMaxSlots - 1) grid = (kMaxSlots - 1) / 8 * 8;
 
   int phases = 0;
   unsigned int panels_before = 0;
@@ -1183,7 +1362,7 @@ cudaError_t launch_chain(const ChainStep* steps, int count, int M, void* workspa
     if ((long long)f.chunks + (long long)q.panels * q.ng > 0x7FFFFFFFLL / 512) return cudaErrorInvalidValue;
     f.chunks += q.panels * q.ng;
     f.last = j + 1;
-    panels_before += (unsigned)q.panels;
+    panels_before += (unsigned)q.panels * kPanelTiles;
   }
   p.phases = phases;
   for (int i = 0; i < phases; ++i) {
@@ -1198,25 +1377,27 @@ cudaError_t launch_chain(const ChainStep* steps, int count, int M, void* workspa
       if (q.panels < grid) {
         int slices = grid / q.panels < q.ng ? grid / q.panels : q.ng;
         if (slices == 2 && q.ng <= 16) slices = 1;
+        // in a cluster launch the CTAs of a panel are 2, 4 or 8 neighbours of one cluster
+        if (p.cluster > 1) slices = slices >= 8 ? 8 : (slices >= 4 ? 4 : (slices >= 2 ? 2 : 1));
         f.unit = -slices;
       }
       // tl_e0m4_tuning_set("decode_split" / "decode_slices") force the cut, as for a lone problem
       if (tune(kTuneDecodeSplit) == 1) f.unit = q.ng;
       if (tune(kTuneDecodeSplit) == 2) f.unit = 1;
       const int64_t forced = tune(kTuneDecodeSlices);
-      if (forced >= 1 && forced <= q.ng && forced * q.panels <= grid) f.unit = -(int)forced;
+      if (forced >= 1 && forced <= q.ng && forced * q.panels <= grid &&
+          (p.cluster == 1 || forced == 1 || forced == 2 || forced == 4 || forced == 8))
+        f.unit = -(int)forced;
     }
   }
-  e = rot ? chain_kernel_launch<true, G>(p, grid, smem, stream) : chain_kernel_launch<false, G>(p, grid, smem, stream);
+  const cudaError_t e =
+      rot ? chain_kernel_launch<true, G>(p, grid, smem, stream) : chain_kernel_launch<false, G>(p, grid, smem, stream);
   count_launch();
   return e;
 }
 
 }  // namespace
 
-#ifdef TL_CHAIN_TRACE
-extern "C" void tl_debug_trace(unsigned long long* out) { cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * 8 * 256); }
-#endif
 size_t decode_chain_workspace_bytes() { return (size_t)kMaxSlots * kSlotBytes + 256; }
 
 cudaError_t launch_gemv_decode_chain(const ChainStep* steps, int count, int M, void* workspace, cudaStream_t stream,

@@ -22,6 +22,7 @@ enum TuneKey {
   kTuneSkipCopies,        // "skip_copies": 1 = the producers of the matmul kernels issue no copies
                           //   (with a short wait limit: makes every bounded wait run out, faulting nothing)
   kTuneRegisterMaxM,      // "register_max_m": most tokens (1..16) a single call gives to the register-fragment kernel
+  kTuneDecodeCluster,     // "decode_cluster": 0 = CTAs that share a panel meet in the global scratch, never in a cluster
   kTuneCount
 };
 
