@@ -302,73 +302,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
     const int jg = (warp - kFirstDequantWarp) >> 2;     // this warp group takes stages jg, jg + 4, ...
     const int n = quad * 32 + lane;                     // weight column of the panel = operand row
     const int t_tile = n >> 4;
-    // 4-bit tiles: a column's 64 bytes are consecutive; 8-bit tiles: chunks of 16 rows, 16 bytes per column
-    const uint32_t pk_off = t_tile * kTileB + (n & 15) * (BITS == 8 ? 16 : 64);
     const uint32_t mask_lo = reg_const(kMaskLo), exp_lo = reg_const(kExpLo);
     const uint32_t mask_hi = reg_const(kMaskHi), exp_hi = reg_const(kExpHi);
-    const __half2 off_lo = __float2half2_rn(126.0f), off_hi = __float2half2_rn(6.0f);
     int it = 0;                  // running stage counter over all items
     int ps = 0, pphase = 0;      // packed ring position of the current group
     for (int item = unit; item < total_items && ok; item += units) {
       const TcItem wi = tc_item<SPLIT, PAIR>(p, item, rank);
       const int R = wi.R;
       for (int g = wi.g0; g < wi.g1 && ok; ++g) {
-        // 64 k of this thread's column: expand, dequantize and write one operand row of 32 columns
         auto expand_half = [&](uint32_t pk, int h, uint32_t taddr) {
-          uint32_t out[32];
-          if (t_tile < R) {
-            __half2 d2, b_lo, b_hi;
-            auto load_scale = [&](int sub) {  // the scale word of group row `sub` of the tile
-              const uint32_t sc = ptx::lds32(pk + kCodeBytes + ((t_tile * kSubs + sub) * 16 + (n & 15)) * 4);
-              const __half2 db = *reinterpret_cast<const __half2*>(&sc);  // {d, b}
-              const __half2 b2 = __high2half2(db);
-              d2 = __low2half2(db);
-              b_lo = __hadd2(b2, off_lo);  // bias seen from the [128, 256) binade (exact)
-              b_hi = __hadd2(b2, off_hi);  // bias seen from the [8, 16) binade (exact)
-            };
-            load_scale(h * 64 / G);
-            if constexpr (BITS == 8) {
-              // 64 codes = 64 bytes; a register of four codes gives two operand words
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                const uint4 wv = ptx::lds128(pk + pk_off + (h * 4 + v) * 256);
-                const uint32_t words[4] = {wv.x, wv.y, wv.z, wv.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint32_t e01 = __byte_perm(words[j], 0x48484848u, 0x4140u);  // {8 + q0 / 128, 8 + q1 / 128}
-                  uint32_t e23 = __byte_perm(words[j], 0x48484848u, 0x4342u);
-                  const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_hi), d2);
-                  const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
-                  out[8 * v + 2 * j + 0] = *reinterpret_cast<const uint32_t*>(&r01);
-                  out[8 * v + 2 * j + 1] = *reinterpret_cast<const uint32_t*>(&r23);
-                }
-              }
-            } else {
-            const uint4 wa = ptx::lds128(pk + pk_off + h * 32);
-            const uint4 wb = ptx::lds128(pk + pk_off + h * 32 + 16);
-            const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-            for (int v = 0; v < 8; ++v) {
-              if (G == 32 && v == 4) load_scale(2 * h + 1);
-              const uint32_t w = words[v], w2 = w >> 8;
-              uint32_t e01 = and_or(w, mask_lo, exp_lo), e23 = and_or(w, mask_hi, exp_hi);
-              uint32_t e45 = and_or(w2, mask_lo, exp_lo), e67 = and_or(w2, mask_hi, exp_hi);
-              const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_lo), d2);
-              const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
-              const __half2 r45 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e45), b_lo), d2);
-              const __half2 r67 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e67), b_hi), d2);
-              out[4 * v + 0] = *reinterpret_cast<const uint32_t*>(&r01);
-              out[4 * v + 1] = *reinterpret_cast<const uint32_t*>(&r23);
-              out[4 * v + 2] = *reinterpret_cast<const uint32_t*>(&r45);
-              out[4 * v + 3] = *reinterpret_cast<const uint32_t*>(&r67);
-            }
-            }
-          } else {
-#pragma unroll
-            for (int v = 0; v < 32; ++v) out[v] = 0u;
-          }
-          // one row of the operand: lane = weight column, 32 columns = 64 consecutive k
-          tmem_st_32x32(taddr, out);
+          expand_half_to_tmem<G, BITS>(pk, h, taddr, t_tile, R, n, mask_lo, exp_lo, mask_hi, exp_hi);
         };
         for (int h = 0; h < 2; h += HALVES, ++it) {
           if ((it & 3) != jg) continue;

@@ -260,10 +260,8 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
     const int jg = (warp - kFirstDequantWarp) >> 2;     // this warp group takes rounds jg, jg + kBatchGroups, ...
     const int n = quad * 32 + lane;                     // weight column of the panel = operand row
     const int t_tile = n >> 4;
-    const uint32_t pk_off = t_tile * kTileB + (n & 15) * (BITS == 8 ? 16 : 64);
     const uint32_t mask_lo = reg_const(kMaskLo), exp_lo = reg_const(kExpLo);
     const uint32_t mask_hi = reg_const(kMaskHi), exp_hi = reg_const(kExpHi);
-    const __half2 off_lo = __float2half2_rn(126.0f), off_hi = __float2half2_rn(6.0f);
     // This group takes rounds jg, jg + kBatchGroups, ... of the CTA's range; its position in the three rings is
     // kept for the NEXT round it takes, so that the rounds of the other groups cost it nothing.
     int it0 = 0;                 // rounds before the current piece
@@ -273,62 +271,8 @@ gemm_tc_batch_kernel(const __grid_constant__ TcBatchParams p) {
     for (PieceWalk<1> w(p, c0, n_rounds, 0); !w.done() && ok; w.next()) {
       const Piece wi = w.cur();
       const int R = wi.R;
-      // 64 k of this thread's column: expand, dequantize and write one operand row of 32 columns
       auto expand_half = [&](uint32_t pk, int h, uint32_t taddr) {
-        uint32_t out[32];
-        if (t_tile < R) {
-          __half2 d2, b_lo, b_hi;
-          auto load_scale = [&](int sub) {  // the scale word of group row `sub` of the tile
-            const uint32_t sc = ptx::lds32(pk + kCodeBytes + ((t_tile * kSubs + sub) * 16 + (n & 15)) * 4);
-            const __half2 db = *reinterpret_cast<const __half2*>(&sc);  // {d, b}
-            const __half2 b2 = __high2half2(db);
-            d2 = __low2half2(db);
-            b_lo = __hadd2(b2, off_lo);  // bias seen from the [128, 256) binade (exact)
-            b_hi = __hadd2(b2, off_hi);  // bias seen from the [8, 16) binade (exact)
-          };
-          load_scale(h * 64 / G);
-          if constexpr (BITS == 8) {
-            // 64 codes = four 16-byte chunks; one byte permute puts two codes into the halves of a
-            // register together with the exponent byte of the binade [8, 16)
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              const uint4 wv = ptx::lds128(pk + pk_off + (h * 4 + v) * 256);
-              const uint32_t words[4] = {wv.x, wv.y, wv.z, wv.w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                uint32_t e01 = __byte_perm(words[j], 0x48484848u, 0x4140u);
-                uint32_t e23 = __byte_perm(words[j], 0x48484848u, 0x4342u);
-                const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_hi), d2);
-                const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
-                out[8 * v + 2 * j + 0] = *reinterpret_cast<const uint32_t*>(&r01);
-                out[8 * v + 2 * j + 1] = *reinterpret_cast<const uint32_t*>(&r23);
-              }
-            }
-          } else {
-          const uint4 wa = ptx::lds128(pk + pk_off + h * 32);
-          const uint4 wb = ptx::lds128(pk + pk_off + h * 32 + 16);
-          const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-          for (int v = 0; v < 8; ++v) {
-            if (G == 32 && v == 4) load_scale(2 * h + 1);
-            const uint32_t wd = words[v], w2 = wd >> 8;
-            uint32_t e01 = and_or(wd, mask_lo, exp_lo), e23 = and_or(wd, mask_hi, exp_hi);
-            uint32_t e45 = and_or(w2, mask_lo, exp_lo), e67 = and_or(w2, mask_hi, exp_hi);
-            const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_lo), d2);
-            const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
-            const __half2 r45 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e45), b_lo), d2);
-            const __half2 r67 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e67), b_hi), d2);
-            out[4 * v + 0] = *reinterpret_cast<const uint32_t*>(&r01);
-            out[4 * v + 1] = *reinterpret_cast<const uint32_t*>(&r23);
-            out[4 * v + 2] = *reinterpret_cast<const uint32_t*>(&r45);
-            out[4 * v + 3] = *reinterpret_cast<const uint32_t*>(&r67);
-          }
-          }
-        } else {
-#pragma unroll
-          for (int v = 0; v < 32; ++v) out[v] = 0u;
-        }
-        tmem_st_32x32(taddr, out);
+        expand_half_to_tmem<G, BITS>(pk, h, taddr, t_tile, R, n, mask_lo, exp_lo, mask_hi, exp_hi);
       };
       const int n_piece = wi.g1 - wi.g0;
       for (; next < it0 + n_piece && ok; next += kBatchGroups) {
@@ -666,10 +610,8 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
     const int jg = (warp - kFirstDequantWarp) >> 2;     // this warp group takes rounds jg, jg + kBatchGroups, ...
     const int n = quad * 32 + lane;                     // weight column of the panel = operand row
     const int t_tile = n >> 4;
-    const uint32_t pk_off = t_tile * kTileB + (n & 15) * (BITS == 8 ? 16 : 64);
     const uint32_t mask_lo = reg_const(kMaskLo), exp_lo = reg_const(kExpLo);
     const uint32_t mask_hi = reg_const(kMaskHi), exp_hi = reg_const(kExpHi);
-    const __half2 off_lo = __float2half2_rn(126.0f), off_hi = __float2half2_rn(6.0f);
     // This group takes rounds jg, jg + kBatchGroups, ... of the CTA's range; its position in the three rings is
     // kept for the NEXT round it takes, so that the rounds of the other groups cost it nothing.
     int it0 = 0;                 // rounds before the current piece
@@ -679,60 +621,8 @@ gemm_tc_batch_pair_kernel(const __grid_constant__ TcBatchParams p) {
     for (PieceWalk<kStep> w(p, c0, n_rounds, rank); !w.done() && ok; w.next()) {
       const Piece wi = w.cur();
       const int R = wi.R;
-      // 64 k of this thread's column: expand, dequantize and write one operand row of 32 columns
       auto expand_half = [&](uint32_t pk, int h, uint32_t taddr) {
-        uint32_t out[32];
-        if (t_tile < R) {
-          __half2 d2, b_lo, b_hi;
-          auto load_scale = [&](int sub) {  // the scale word of group row `sub` of the tile
-            const uint32_t sc = ptx::lds32(pk + kCodeBytes + ((t_tile * kSubs + sub) * 16 + (n & 15)) * 4);
-            const __half2 db = *reinterpret_cast<const __half2*>(&sc);  // {d, b}
-            const __half2 b2 = __high2half2(db);
-            d2 = __low2half2(db);
-            b_lo = __hadd2(b2, off_lo);  // bias seen from the [128, 256) binade (exact)
-            b_hi = __hadd2(b2, off_hi);  // bias seen from the [8, 16) binade (exact)
-          };
-          load_scale(h * 64 / G);
-          if constexpr (BITS == 8) {
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              const uint4 wv = ptx::lds128(pk + pk_off + (h * 4 + v) * 256);
-              const uint32_t words[4] = {wv.x, wv.y, wv.z, wv.w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                uint32_t e01 = __byte_perm(words[j], 0x48484848u, 0x4140u);
-                uint32_t e23 = __byte_perm(words[j], 0x48484848u, 0x4342u);
-                const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_hi), d2);
-                const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
-                out[8 * v + 2 * j + 0] = *reinterpret_cast<const uint32_t*>(&r01);
-                out[8 * v + 2 * j + 1] = *reinterpret_cast<const uint32_t*>(&r23);
-              }
-            }
-          } else {
-          const uint4 wa = ptx::lds128(pk + pk_off + h * 32);
-          const uint4 wb = ptx::lds128(pk + pk_off + h * 32 + 16);
-          const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-          for (int v = 0; v < 8; ++v) {
-            if (G == 32 && v == 4) load_scale(2 * h + 1);
-            const uint32_t wd = words[v], w2 = wd >> 8;
-            uint32_t e01 = and_or(wd, mask_lo, exp_lo), e23 = and_or(wd, mask_hi, exp_hi);
-            uint32_t e45 = and_or(w2, mask_lo, exp_lo), e67 = and_or(w2, mask_hi, exp_hi);
-            const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_lo), d2);
-            const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
-            const __half2 r45 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e45), b_lo), d2);
-            const __half2 r67 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e67), b_hi), d2);
-            out[4 * v + 0] = *reinterpret_cast<const uint32_t*>(&r01);
-            out[4 * v + 1] = *reinterpret_cast<const uint32_t*>(&r23);
-            out[4 * v + 2] = *reinterpret_cast<const uint32_t*>(&r45);
-            out[4 * v + 3] = *reinterpret_cast<const uint32_t*>(&r67);
-          }
-          }
-        } else {
-#pragma unroll
-          for (int v = 0; v < 32; ++v) out[v] = 0u;
-        }
-        tmem_st_32x32(taddr, out);
+        expand_half_to_tmem<G, BITS>(pk, h, taddr, t_tile, R, n, mask_lo, exp_lo, mask_hi, exp_hi);
       };
       const int n_piece = wi.g1 - wi.g0;
       for (; next < it0 + n_piece && ok; next += kBatchGroups) {

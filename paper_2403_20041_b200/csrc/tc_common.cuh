@@ -4,6 +4,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ptx.cuh"
 #include "umma.cuh"
 
 namespace tl {
@@ -47,6 +48,79 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
       "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
       "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
+}
+
+// The dequantizer of the tensor-core kernels: 64 k of one weight column (thread = column n of the
+// panel, `h` = which half of the 128-k round) are expanded from the packed slot at shared address
+// `pk`, dequantized exactly as the standalone dequantizer does, (w1 - b) * d with the bias seen
+// from the binade the code was completed in, and written as one operand row of 32 tensor-memory
+// columns at `taddr`.  Columns of a ragged panel beyond its last tile (t_tile >= R) are fed zeros.
+// 4-bit tiles: a column's 64 bytes are consecutive; 8-bit tiles: chunks of 16 rows, 16 bytes per
+// column, and one byte permute puts two codes into the halves of a register together with the
+// exponent byte of the binade [8, 16).
+template <int G, int BITS>
+__device__ __forceinline__ void expand_half_to_tmem(uint32_t pk, int h, uint32_t taddr, int t_tile, int R, int n,
+                                                    uint32_t mask_lo, uint32_t exp_lo, uint32_t mask_hi,
+                                                    uint32_t exp_hi) {
+  constexpr int kSubs = kGroup / G;                       // scale words per column and tile row
+  constexpr int kTileB = BITS == 8 ? 2048 : 1024;         // bytes of a packed tile (16 columns x 128 k)
+  constexpr int kCodeBytes = kPanelTiles * kTileB;        // codes of a slot; the scale words follow them
+  const uint32_t pk_off = t_tile * kTileB + (n & 15) * (BITS == 8 ? 16 : 64);
+  const __half2 off_lo = __float2half2_rn(126.0f), off_hi = __float2half2_rn(6.0f);
+  uint32_t out[32];
+  if (t_tile < R) {
+    __half2 d2, b_lo, b_hi;
+    auto load_scale = [&](int sub) {  // the scale word of group row `sub` of the tile
+      const uint32_t sc = ptx::lds32(pk + kCodeBytes + ((t_tile * kSubs + sub) * 16 + (n & 15)) * 4);
+      const __half2 db = *reinterpret_cast<const __half2*>(&sc);  // {d, b}
+      const __half2 b2 = __high2half2(db);
+      d2 = __low2half2(db);
+      b_lo = __hadd2(b2, off_lo);  // bias seen from the [128, 256) binade (exact)
+      b_hi = __hadd2(b2, off_hi);  // bias seen from the [8, 16) binade (exact)
+    };
+    load_scale(h * 64 / G);
+    if constexpr (BITS == 8) {
+      // 64 codes = four 16-byte chunks; a register of four codes gives two operand words
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const uint4 wv = ptx::lds128(pk + pk_off + (h * 4 + v) * 256);
+        const uint32_t words[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t e01 = __byte_perm(words[j], 0x48484848u, 0x4140u);  // {8 + q0 / 128, 8 + q1 / 128}
+          uint32_t e23 = __byte_perm(words[j], 0x48484848u, 0x4342u);
+          const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_hi), d2);
+          const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
+          out[8 * v + 2 * j + 0] = *reinterpret_cast<const uint32_t*>(&r01);
+          out[8 * v + 2 * j + 1] = *reinterpret_cast<const uint32_t*>(&r23);
+        }
+      }
+    } else {
+      const uint4 wa = ptx::lds128(pk + pk_off + h * 32);
+      const uint4 wb = ptx::lds128(pk + pk_off + h * 32 + 16);
+      const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {
+        if (G == 32 && v == 4) load_scale(2 * h + 1);
+        const uint32_t w = words[v], w2 = w >> 8;
+        uint32_t e01 = and_or(w, mask_lo, exp_lo), e23 = and_or(w, mask_hi, exp_hi);
+        uint32_t e45 = and_or(w2, mask_lo, exp_lo), e67 = and_or(w2, mask_hi, exp_hi);
+        const __half2 r01 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e01), b_lo), d2);
+        const __half2 r23 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e23), b_hi), d2);
+        const __half2 r45 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e45), b_lo), d2);
+        const __half2 r67 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e67), b_hi), d2);
+        out[4 * v + 0] = *reinterpret_cast<const uint32_t*>(&r01);
+        out[4 * v + 1] = *reinterpret_cast<const uint32_t*>(&r23);
+        out[4 * v + 2] = *reinterpret_cast<const uint32_t*>(&r45);
+        out[4 * v + 3] = *reinterpret_cast<const uint32_t*>(&r67);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int v = 0; v < 32; ++v) out[v] = 0u;
+  }
+  // one row of the operand: lane = weight column, 32 columns = 64 consecutive k
+  tmem_st_32x32(taddr, out);
 }
 
 // D[tmem] (+)= A[tmem] * B[smem]: A is read from tensor memory (row = lane, two fp16 per column).

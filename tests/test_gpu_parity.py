@@ -660,3 +660,35 @@ def test_list_kernel_with_and_without_paired_ctas(lib, dev, tuning, pair, M):
         assert np.isfinite(y_np).all()
         assert_matmul_close(y_np[:, cols], y_ref)
     assert lib.tl_e0m4_device_status() == 0
+
+
+# ---------------------------------------------------------------- panels shared by a cluster of CTAs
+@pytest.mark.parametrize("cluster", [0, 1])
+@pytest.mark.parametrize("group", [128, 32])
+@pytest.mark.parametrize("M", [1, 5, 8])
+def test_shared_panels_meet_in_scratch_or_in_a_cluster(lib, dev, tuning, M, group, cluster):
+    """The CTAs that share a panel's k groups add their partial sums up either in the global scratch
+    (cluster = 0) or, launched as a thread-block cluster, in one another's shared memory (1: forced
+    wherever the shape allows it).  2128 columns: sixteen full panels and one of five column blocks,
+    so some CTAs of the last cluster have no tile to finish.  Plain, residual and SwiGLU epilogues."""
+    tuning("decode_cluster", cluster)
+    K, N = 2048, 2128
+    w_np = workloads.weights(K, N, seed=workloads.seed_for("cluster", group))
+    x_np = workloads.activations(M, K, seed=workloads.seed_for("cluster", "x", M))
+    r_np = workloads.activations(M, N, seed=workloads.seed_for("cluster", "r", M))
+    codes, d_h, b_h = oracle.quantize(w_np, group=group)
+    w_hat = oracle.dequantize(codes, d_h, b_h, group=group)
+    packed, scales = lib.tl_e0m4_quantize(torch.from_numpy(w_np).to(dev), group=group)
+    x, r = torch.from_numpy(x_np).to(dev), torch.from_numpy(r_np).to(dev)
+    ws = lib.tl_e0m4_workspace(lib.tl_e0m4_matmul_workspace(M, K, N), dev)
+    for _ in range(2):
+        y = lib.tl_e0m4_matmul(x, packed, scales, N, workspace=ws, group=group)
+        y_add = lib.tl_e0m4_matmul_add(x, packed, scales, N, r, y=torch.empty_like(r), workspace=ws, group=group)
+        y_glu = lib.tl_e0m4_matmul_swiglu(x, packed, scales, N, workspace=ws, group=group)
+        torch.cuda.synchronize()
+        assert not _to_np(ws).any()
+        y_ref = oracle.matmul(x_np, w_hat)
+        assert_matmul_close(_to_np(y), y_ref)
+        assert_matmul_close(_to_np(y_add), oracle.matmul(x_np, w_hat, addend_h=r_np))
+        assert_matmul_close(_to_np(y_glu), oracle.swiglu_blocks(y_ref))
+    assert lib.tl_e0m4_device_status() == 0
