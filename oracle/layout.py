@@ -27,6 +27,13 @@ be compared bit for bit:
 2048 bytes, made of eight chunks of 256 bytes, one per 16 rows; in chunk (k % 128) // 16 column
 n % 16 owns 16 consecutive bytes and byte k % 16 of them is the code of row k.  The
 coefficient words do not change.
+
+3-bit and 5-bit codes (``bits=3``, ``bits=5``): the same tiles in the same order.  Eight
+consecutive k of one column form a unit of ``bits`` bytes, read as a little-endian integer in
+which the code of k % 8 = c occupies bits c * bits .. (c + 1) * bits - 1.  Inside a tile column
+n % 16 owns its 16 units one after the other (16 * bits bytes), so a tile is 256 * bits bytes and
+the 128 codes of a column's tile row are one continuous little-endian bit string: the code of row
+k starts at bit (k % 128) * bits of it.  The coefficient words do not change.
 """
 
 from __future__ import annotations
@@ -40,8 +47,8 @@ PANEL_TILES = 8
 
 def packed_sizes(K: int, N: int, group: int = TILE_K, bits: int = 4):
     """Bytes of the packed-code buffer and of the coefficient buffer."""
-    if bits not in (4, 8):
-        raise ValueError("the container holds 4-bit or 8-bit codes")
+    if bits not in (3, 4, 5, 8):
+        raise ValueError("the container holds 3-, 4-, 5- or 8-bit codes")
     if K <= 0 or N <= 0 or K % TILE_K or N % TILE_N:
         raise ValueError("K must be a multiple of 128 and N a multiple of 16")
     if group not in (32, 64, 128):
@@ -78,6 +85,15 @@ def _byte_index(K, N):
     return _tile_index(k, n, K, N) * (TILE_N * TILE_K) + chunk * (TILE_N * 16) + (n % TILE_N) * 16 + k % 16
 
 
+def _bit_index(K, N, bits):
+    """Position (in bits from the start of the packed stream) of the lowest bit of every 3- or
+    5-bit code: [K, N]."""
+    k = np.arange(K)[:, None]
+    n = np.arange(N)[None, :]
+    column_start = _tile_index(k, n, K, N) * (256 * bits) + (n % TILE_N) * (16 * bits)  # bytes
+    return column_start * 8 + (k % TILE_K) * bits
+
+
 def pack(codes, d_h, b_h, group: int = TILE_K, bits: int = 4):
     """Logical (codes[K,N] uint8, d_h[K/G,N] fp16, b_h[K/G,N] fp16) ->
     (packed uint32[K*N*bits/32], scales uint32[K/G*N])."""
@@ -91,6 +107,14 @@ def pack(codes, d_h, b_h, group: int = TILE_K, bits: int = 4):
         stream = np.zeros(K * N, dtype=np.uint8)
         stream[_byte_index(K, N).ravel()] = codes.ravel()
         packed = stream.view("<u4").astype(np.uint32)
+    elif bits in (3, 5):
+        # one bit at a time into a stream of single bits, then eight bits to the byte, lowest first
+        stream_bits = np.zeros(K * N * bits, dtype=np.uint8)
+        start = _bit_index(K, N, bits).ravel()
+        flat = codes.ravel()
+        for i in range(bits):
+            stream_bits[start + i] = (flat >> i) & 1
+        packed = np.packbits(stream_bits, bitorder="little").view("<u4").astype(np.uint32)
     else:
         word = _tile_index(k, n, K, N) * 256 + (n % TILE_N) * 16 + (k % TILE_K) // 8
         shift = (4 * _nibble_pos(k % 8)).astype(np.uint32) + np.zeros_like(n, dtype=np.uint32)
@@ -114,6 +138,12 @@ def unpack(packed, scales, K: int, N: int, group: int = TILE_K, bits: int = 4):
     n = np.arange(N)[None, :]
     if bits == 8:
         codes = packed.astype("<u4").view(np.uint8)[_byte_index(K, N)]
+    elif bits in (3, 5):
+        stream_bits = np.unpackbits(packed.astype("<u4").view(np.uint8), bitorder="little")
+        start = _bit_index(K, N, bits)
+        codes = np.zeros((K, N), dtype=np.uint8)
+        for i in range(bits):
+            codes |= (stream_bits[start + i] << i).astype(np.uint8)
     else:
         word = _tile_index(k, n, K, N) * 256 + (n % TILE_N) * 16 + (k % TILE_K) // 8
         shift = (4 * _nibble_pos(k % 8)).astype(np.uint32) + np.zeros_like(n, dtype=np.uint32)
