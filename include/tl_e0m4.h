@@ -367,6 +367,31 @@ tl_status tl_e0m8_matmul_swiglu(const void* x_dev, const void* packed_dev, const
 tl_status tl_e0m8_matmul_batch(const tl_e0m4_problem* problems_host, int count, int64_t M, int group,
                                void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * E0M3 and E0M5: the construction of Section 2.3 with three or five fraction bits kept ("other
+ * bit-width quantization").  `bits` is 3 or 5 (TL_ERR_SHAPE otherwise; 4 and 8 have the entry points
+ * above).  A code is the `bits` highest fraction bits of w1 in [2, 4):
+ * as_half(0x4000 | code << (10 - bits)) = 2 + code / 2^(bits - 1); the steps are those of
+ * tl_e0m4_quantize with 2^bits for 16, 2^bits - 1 for 15 and 2^(bits - 1) for 8.
+ * Container: the 4-bit layout's tiles (16 columns x 128 rows) in the same order; eight consecutive k
+ * of one column are a unit of `bits` bytes, a little-endian integer in which the code of k % 8 = c
+ * occupies bits c * bits .. (c + 1) * bits - 1, and column n % 16 of a tile owns its 16 units one
+ * after the other: byte 256 * bits * tile + 16 * bits * (n % 16) + bits * ((k % 128) / 8) is the
+ * first byte of the unit of row k.  packed_dev holds K * N * bits / 8 bytes; scales_dev is laid
+ * out as for E0M4.  group must be 128.  Other arguments, ownership, alignment rules and errors
+ * are those of the E0M4 entry points of the same name.  tl_e0mx_matmul runs every M on the
+ * tensor-core kernel (plain product; its workspace, tl_e0mx_matmul_workspace(M, K, N, bits) bytes,
+ * possibly 0, is zero on entry and left zero). */
+tl_status tl_e0mx_packed_sizes(int64_t K, int64_t N, int group, int bits, size_t* packed_bytes, size_t* scales_bytes);
+tl_status tl_e0mx_quantize(const void* w_dev, tl_dtype w_dtype, int64_t K, int64_t N, int group, int bits,
+                           void* packed_dev, void* scales_dev, void* stream);
+tl_status tl_e0mx_dequant(const void* packed_dev, const void* scales_dev, int64_t K, int64_t N, int group, int bits,
+                          void* w_f16_dev, void* stream);
+size_t tl_e0mx_matmul_workspace(int64_t M, int64_t K, int64_t N, int bits);
+tl_status tl_e0mx_matmul(const void* x_dev, const void* packed_dev, const void* scales_dev, void* y_dev, int64_t M,
+                         int64_t K, int64_t N, int group, int bits, void* workspace_dev, size_t workspace_bytes,
+                         void* stream);
+
 /* Reads the device status word that kernels set when a bounded device-side wait gives up
  * (TL_ERR_TIMEOUT), clears it, and returns it.  Synchronizes `stream`.  Diagnostics only. */
 tl_status tl_e0m4_device_status(void* stream);

@@ -64,6 +64,11 @@ SYMBOLS = {
     "tl_e0m8_matmul_add": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _sz, _vp]),
     "tl_e0m8_matmul_bias": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _sz, _vp]),
     "tl_e0m8_matmul_swiglu": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _sz, _vp]),
+    "tl_e0mx_packed_sizes": (_int, [_i64, _i64, _int, _int, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
+    "tl_e0mx_quantize": (_int, [_vp, _int, _i64, _i64, _int, _int, _vp, _vp, _vp]),
+    "tl_e0mx_dequant": (_int, [_vp, _vp, _i64, _i64, _int, _int, _vp, _vp]),
+    "tl_e0mx_matmul_workspace": (_sz, [_i64, _i64, _i64, _int]),
+    "tl_e0mx_matmul": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _vp, _sz, _vp]),
     "tl_e0m4_launch_count": (ctypes.c_uint64, []),
     "tl_status_string": (ctypes.c_char_p, [_int]),
 }
@@ -268,6 +273,62 @@ def tl_e0m8_matmul_bias(x, packed, scales, N: int, bias, y=None, workspace=None,
 def tl_e0m8_matmul_swiglu(x, packed, scales, N: int, y=None, workspace=None, group: int = GROUP, stream=None):
     """y[M, N / 2] = silu(gate) * up over column blocks of eight of x . W, for E0M8 weights."""
     return _matmul8("tl_e0m8_matmul_swiglu", x, packed, scales, N, None, y, N // 2, workspace, group, stream)
+
+
+def tl_e0mx_packed_sizes(K: int, N: int, bits: int, group: int = GROUP):
+    """(packed_bytes, scales_bytes) of a [K, N] weight in the 3-bit or 5-bit container."""
+    a, b = _sz(0), _sz(0)
+    _check(lib().tl_e0mx_packed_sizes(K, N, group, bits, ctypes.byref(a), ctypes.byref(b)), "tl_e0mx_packed_sizes")
+    return a.value, b.value
+
+
+def tl_e0mx_quantize(w, bits: int, packed=None, scales=None, group: int = GROUP, stream=None):
+    """Quantize a CUDA weight tensor [K, N] (fp32 or fp16) to E0M3 or E0M5.  Returns (packed, scales)."""
+    import torch
+
+    K, N = w.shape
+    pb, sb = tl_e0mx_packed_sizes(K, N, bits, group)
+    if packed is None:
+        packed = torch.empty(pb, dtype=torch.uint8, device=w.device)
+    if scales is None:
+        scales = torch.empty(sb, dtype=torch.uint8, device=w.device)
+    if w.dtype not in (torch.float32, torch.float16):
+        raise ValueError("weights must be float32 or float16")
+    dt = TL_F32 if w.dtype == torch.float32 else TL_F16
+    _check(lib().tl_e0mx_quantize(_dev_ptr(w, "w"), dt, K, N, group, bits, _dev_ptr(packed, "packed"),
+                                  _dev_ptr(scales, "scales"), _stream(stream)), "tl_e0mx_quantize")
+    return packed, scales
+
+
+def tl_e0mx_dequant(packed, scales, K: int, N: int, bits: int, out=None, group: int = GROUP, stream=None):
+    """Expand E0M3 / E0M5 weights to a dense fp16 [K, N] CUDA tensor."""
+    import torch
+
+    if out is None:
+        out = torch.empty((K, N), dtype=torch.float16, device=packed.device)
+    _check(lib().tl_e0mx_dequant(_dev_ptr(packed, "packed"), _dev_ptr(scales, "scales"), K, N, group, bits,
+                                 _dev_ptr(out, "out"), _stream(stream)), "tl_e0mx_dequant")
+    return out
+
+
+def tl_e0mx_matmul(x, packed, scales, N: int, bits: int, y=None, workspace=None, group: int = GROUP, stream=None):
+    """y[M, N] = x[M, K] . W with W in packed E0M3 / E0M5 form (fp16 in/out, fp32 accumulation)."""
+    import torch
+
+    M, K = x.shape
+    if x.dtype != torch.float16:
+        raise ValueError("x must be float16")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=x.device)
+    need = int(lib().tl_e0mx_matmul_workspace(M, K, N, bits))
+    if need and workspace is None:
+        workspace = tl_e0m4_workspace(need, x.device, stream=stream)
+    ws_ptr = _dev_ptr(workspace, "workspace") if workspace is not None else None
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(lib().tl_e0mx_matmul(_dev_ptr(x, "x"), _dev_ptr(packed, "packed"), _dev_ptr(scales, "scales"),
+                                _dev_ptr(y, "y"), M, K, N, group, bits, ws_ptr, ws_bytes, _stream(stream)),
+           "tl_e0mx_matmul")
+    return y
 
 
 def tl_kv_append(cache, new, position_ids, stream=None):

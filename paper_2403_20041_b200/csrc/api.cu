@@ -264,6 +264,75 @@ tl_status tl_e0m8_matmul_batch(const tl_e0m4_problem* problems_host, int count, 
   return TL_OK;
 }
 
+// ---------------------------------------------------------------- E0M3 / E0M5 (three or five fraction bits kept)
+
+tl_status tl_e0mx_packed_sizes(int64_t K, int64_t N, int group, int bits, size_t* packed_bytes, size_t* scales_bytes) {
+  if (group != kGroup || (bits != 3 && bits != 5)) return TL_ERR_SHAPE;
+  const tl_status st = check_shape(K, N, group);
+  if (st != TL_OK) return st;
+  if (packed_bytes) *packed_bytes = (size_t)K * (size_t)N * (size_t)bits / 8;
+  if (scales_bytes) *scales_bytes = (size_t)(K / group) * (size_t)N * 4;
+  return TL_OK;
+}
+
+tl_status tl_e0mx_quantize(const void* w_dev, tl_dtype w_dtype, int64_t K, int64_t N, int group, int bits,
+                           void* packed_dev, void* scales_dev, void* stream) {
+  if (!w_dev || !packed_dev || !scales_dev) return TL_ERR_NULL;
+  if (w_dtype != TL_F32 && w_dtype != TL_F16) return TL_ERR_DTYPE;
+  if (group != kGroup || (bits != 3 && bits != 5)) return TL_ERR_SHAPE;
+  tl_status st = check_shape(K, N, group);
+  if (st != TL_OK) return st;
+  if (!aligned16(w_dev) || !aligned16(packed_dev) || !aligned16(scales_dev)) return TL_ERR_ALIGN;
+  if ((st = check_device()) != TL_OK) return st;
+  const cudaError_t e = launch_quantize_x(w_dev, w_dtype, K, N, bits, static_cast<uint8_t*>(packed_dev),
+                                          static_cast<uint32_t*>(scales_dev), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TL_OK : TL_ERR_CUDA;
+}
+
+tl_status tl_e0mx_dequant(const void* packed_dev, const void* scales_dev, int64_t K, int64_t N, int group, int bits,
+                          void* w_f16_dev, void* stream) {
+  if (!packed_dev || !scales_dev || !w_f16_dev) return TL_ERR_NULL;
+  if (group != kGroup || (bits != 3 && bits != 5)) return TL_ERR_SHAPE;
+  tl_status st = check_shape(K, N, group);
+  if (st != TL_OK) return st;
+  if (!aligned16(packed_dev) || !aligned16(scales_dev) || !aligned16(w_f16_dev)) return TL_ERR_ALIGN;
+  if ((st = check_device()) != TL_OK) return st;
+  const cudaError_t e =
+      launch_dequant_x(static_cast<const uint8_t*>(packed_dev), static_cast<const uint32_t*>(scales_dev), K, N, bits,
+                       static_cast<__half*>(w_f16_dev), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TL_OK : TL_ERR_CUDA;
+}
+
+size_t tl_e0mx_matmul_workspace(int64_t M, int64_t K, int64_t N, int bits) {
+  if (M <= 0 || K <= 0 || N <= 0 || K % kGroup != 0 || N % kTileN != 0 || (bits != 3 && bits != 5)) return 0;
+  return gemm_tc_workspace_bytes(M, K, N, bits);
+}
+
+tl_status tl_e0mx_matmul(const void* x_dev, const void* packed_dev, const void* scales_dev, void* y_dev, int64_t M,
+                         int64_t K, int64_t N, int group, int bits, void* workspace_dev, size_t workspace_bytes,
+                         void* stream) {
+  if (!x_dev || !packed_dev || !scales_dev || !y_dev) return TL_ERR_NULL;
+  if (group != kGroup || (bits != 3 && bits != 5)) return TL_ERR_SHAPE;
+  tl_status st = check_shape(K, N, group);
+  if (st != TL_OK) return st;
+  if (M <= 0 || M > (int64_t)1 << 20) return TL_ERR_SHAPE;
+  if (!aligned16(x_dev) || !aligned16(packed_dev) || !aligned16(scales_dev) || !aligned16(y_dev)) return TL_ERR_ALIGN;
+  const size_t need = tl_e0mx_matmul_workspace(M, K, N, bits);
+  if (need > 0) {
+    if (!workspace_dev || workspace_bytes < need) return TL_ERR_WORKSPACE;
+    if (!aligned16(workspace_dev)) return TL_ERR_ALIGN;
+  }
+  if ((st = check_device()) != TL_OK) return st;
+  unsigned int* status = device_status_ptr();
+  if (!status) return TL_ERR_CUDA;
+  // every M runs on the tensor-core kernel, as for E0M8
+  const cudaError_t e =
+      launch_gemm_tc(static_cast<const __half*>(x_dev), static_cast<const uint32_t*>(packed_dev),
+                     static_cast<const uint32_t*>(scales_dev), static_cast<__half*>(y_dev), M, K, N, workspace_dev,
+                     status, static_cast<cudaStream_t>(stream), nullptr, false, kGroup, -1, bits);
+  return e == cudaSuccess ? TL_OK : TL_ERR_CUDA;
+}
+
 tl_kernel tl_e0m4_matmul_kernel(int64_t M, int64_t K, int64_t N) {
   (void)K;
   (void)N;

@@ -126,6 +126,12 @@ cudaError_t launch_quantize8(const void* w, tl_dtype dt, int64_t K, int64_t N, u
                              cudaStream_t stream);
 cudaError_t launch_dequant8(const uint8_t* packed, const uint32_t* scales, int64_t K, int64_t N, __half* out,
                             cudaStream_t stream);
+// E0M3 / E0M5 (three or five fraction bits kept, units of eight codes in `bits` bytes, groups of 128):
+// quantizer and dequantizer; the matmul is launch_gemm_tc with bits = 3 or 5 (plain epilogue), for every M.
+cudaError_t launch_quantize_x(const void* w, tl_dtype dt, int64_t K, int64_t N, int bits, uint8_t* packed,
+                              uint32_t* scales, cudaStream_t stream);
+cudaError_t launch_dequant_x(const uint8_t* packed, const uint32_t* scales, int64_t K, int64_t N, int bits, __half* out,
+                             cudaStream_t stream);
 // Tensor-core kernel over a list of independent problems that share M (at most kMaxTcBatchM tokens;
 // longer lists take several launches).  `workspace` holds gemm_tc_batch_workspace_bytes() bytes, zero
 // on entry and left zero.

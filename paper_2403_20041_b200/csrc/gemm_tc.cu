@@ -124,10 +124,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
   static_assert(!(PAIR && BIG), "pairs work in 64-k rounds");
   constexpr int HALVES = BIG ? 2 : 1;  // 64-k halves per round
   constexpr int kSubs = kGroup / G;    // scale words per column and tile row
-  static_assert(BITS == 4 || (BITS == 8 && G == kGroup), "8-bit codes come with groups of 128");
-  constexpr int kTileB = BITS == 8 ? 2048 : 1024;   // bytes of a packed tile (16 columns x 128 k)
+  static_assert(BITS == 4 || ((BITS == 8 || BITS == 3 || BITS == 5) && G == kGroup), "other widths come with groups of 128");
+  constexpr int kTileB = 256 * BITS;                // bytes of a packed tile (16 columns x 128 k)
   constexpr int kCodeBytes = kPanelTiles * kTileB;  // codes of a slot; the scale words follow them
-  constexpr int kSlot = BITS == 8 ? tc_slot_bytes(8, G) : packed_slot_bytes(G);
+  constexpr int kSlot = tc_slot_bytes(BITS, G);
   const int S = p.sx;
   const int rank = PAIR ? (int)(blockIdx.x & 1u) : 0;              // CTA rank in the cluster of two
   const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;  // index of the CTA (pair) among its peers
@@ -776,11 +776,16 @@ cudaError_t launch_gemm_tc(const __half* x, const uint32_t* packed, const uint32
   auto launch_epi = [&](auto epi) {
     constexpr std::integral_constant<int, 4> four{};
     if (bits == 8) return launch_group(epi, std::integral_constant<int, kGroup>{}, std::integral_constant<int, 8>{});
+    if constexpr (decltype(epi)::value == 0) {  // 3-bit and 5-bit codes: the plain product only
+      if (bits == 3) return launch_group(epi, std::integral_constant<int, kGroup>{}, std::integral_constant<int, 3>{});
+      if (bits == 5) return launch_group(epi, std::integral_constant<int, kGroup>{}, std::integral_constant<int, 5>{});
+    }
+    if (bits != 4) return cudaErrorInvalidValue;
     if (group == 32) return launch_group(epi, std::integral_constant<int, 32>{}, four);
     if (group == 64) return launch_group(epi, std::integral_constant<int, 64>{}, four);
     return launch_group(epi, std::integral_constant<int, 128>{}, four);
   };
-  if (bits == 8 && group != kGroup) return cudaErrorInvalidValue;
+  if (bits != 4 && group != kGroup) return cudaErrorInvalidValue;
   if (add) e = launch_epi(std::integral_constant<int, 1>{});
   else if (swiglu) e = launch_epi(std::integral_constant<int, 2>{});
   else e = launch_epi(std::integral_constant<int, 0>{});

@@ -19,9 +19,10 @@ constexpr int kMaxPackedSlots = 24;
 // a slot of the packed ring: 8 KB codes + the scale words of 128 k (512 B per group row of the
 // tile), padded to a multiple of 1024
 __host__ __device__ constexpr int packed_slot_bytes(int group) { return 8192 + (512 * (kGroup / group) + 1023) / 1024 * 1024; }
-// the same for either code width: 8-bit codes take 16 KB per 128 k of a panel
+// the same for every code width: 8-bit codes take 16 KB per 128 k of a panel, 3-bit and 5-bit
+// codes 6 KB and 10 KB (groups of 128 only), each followed by 1 KB for the scale words
 __host__ __device__ constexpr int tc_slot_bytes(int bits, int group) {
-  return bits == 8 ? 16384 + 1024 : packed_slot_bytes(group);
+  return bits == 4 ? packed_slot_bytes(group) : kPanelTiles * 256 * bits + 1024;
 }
 constexpr int kPackedSlotBytes = packed_slot_bytes(kGroup);
 constexpr int kPackedOffset = kXRingBytes;
@@ -57,23 +58,25 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
 // columns at `taddr`.  Columns of a ragged panel beyond its last tile (t_tile >= R) are fed zeros.
 // 4-bit tiles: a column's 64 bytes are consecutive; 8-bit tiles: chunks of 16 rows, 16 bytes per
 // column, and one byte permute puts two codes into the halves of a register together with the
-// exponent byte of the binade [8, 16).
+// exponent byte of the binade [8, 16).  3-bit and 5-bit tiles: a column's 128 codes are one little-endian
+// bit string of 16 * bits bytes; the codes are cut out of it with funnel shifts and completed in the
+// binade [2, 4) itself (shift 10 - bits), as the formula of Section 2.3 has it.
 template <int G, int BITS>
 __device__ __forceinline__ void expand_half_to_tmem(uint32_t pk, int h, uint32_t taddr, int t_tile, int R, int n,
                                                     uint32_t mask_lo, uint32_t exp_lo, uint32_t mask_hi,
                                                     uint32_t exp_hi) {
   constexpr int kSubs = kGroup / G;                       // scale words per column and tile row
-  constexpr int kTileB = BITS == 8 ? 2048 : 1024;         // bytes of a packed tile (16 columns x 128 k)
+  constexpr int kTileB = 256 * BITS;                      // bytes of a packed tile (16 columns x 128 k)
   constexpr int kCodeBytes = kPanelTiles * kTileB;        // codes of a slot; the scale words follow them
-  const uint32_t pk_off = t_tile * kTileB + (n & 15) * (BITS == 8 ? 16 : 64);
+  const uint32_t pk_off = t_tile * kTileB + (n & 15) * (BITS == 8 ? 16 : 16 * BITS);
   const __half2 off_lo = __float2half2_rn(126.0f), off_hi = __float2half2_rn(6.0f);
   uint32_t out[32];
   if (t_tile < R) {
-    __half2 d2, b_lo, b_hi;
+    __half2 d2, b2, b_lo, b_hi;
     auto load_scale = [&](int sub) {  // the scale word of group row `sub` of the tile
       const uint32_t sc = ptx::lds32(pk + kCodeBytes + ((t_tile * kSubs + sub) * 16 + (n & 15)) * 4);
       const __half2 db = *reinterpret_cast<const __half2*>(&sc);  // {d, b}
-      const __half2 b2 = __high2half2(db);
+      b2 = __high2half2(db);
       d2 = __low2half2(db);
       b_lo = __hadd2(b2, off_lo);  // bias seen from the [128, 256) binade (exact)
       b_hi = __hadd2(b2, off_hi);  // bias seen from the [8, 16) binade (exact)
@@ -94,6 +97,21 @@ __device__ __forceinline__ void expand_half_to_tmem(uint32_t pk, int h, uint32_t
           out[8 * v + 2 * j + 0] = *reinterpret_cast<const uint32_t*>(&r01);
           out[8 * v + 2 * j + 1] = *reinterpret_cast<const uint32_t*>(&r23);
         }
+      }
+    } else if constexpr (BITS == 3 || BITS == 5) {
+      constexpr int kW = 64 * BITS / 32;  // words of this half of the column's bit string
+      uint32_t wds[kW + 1];
+#pragma unroll
+      for (int i = 0; i < kW; ++i) wds[i] = ptx::lds32(pk + pk_off + h * (8 * BITS) + 4 * i);
+      wds[kW] = 0u;
+#pragma unroll
+      for (int c = 0; c < 64; c += 2) {
+        const int at0 = c * BITS, at1 = at0 + BITS;
+        const uint32_t q0 = __funnelshift_r(wds[at0 >> 5], wds[(at0 >> 5) + 1], at0 & 31) & ((1u << BITS) - 1u);
+        const uint32_t q1 = __funnelshift_r(wds[at1 >> 5], wds[(at1 >> 5) + 1], at1 & 31) & ((1u << BITS) - 1u);
+        uint32_t e = 0x40004000u | (q0 << (10 - BITS)) | (q1 << (26 - BITS));  // {2 + q0 / 2^(bits-1), 2 + q1 / ...}
+        const __half2 r = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&e), b2), d2);
+        out[c >> 1] = *reinterpret_cast<const uint32_t*>(&r);
       }
     } else {
       const uint4 wa = ptx::lds128(pk + pk_off + h * 32);
