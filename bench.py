@@ -543,6 +543,37 @@ def bench_e0m8(binding, workloads, torch, dev, peaks, tokens=(1, 4, 16, 64, 128,
     return out
 
 
+def bench_e0mx(binding, workloads, torch, dev, peaks):
+    """E0M3 and E0M5 (the construction of Section 2.3 with three or five fraction bits kept; bits / 8 + 4 / 128
+    bytes per weight): mean absolute error, quantizer and dequantizer rates on a 4096 x 27392 matrix and the
+    tensor-core matmul on it at 16 and 2048 tokens."""
+    K, N = 4096, 27392
+    w = workloads.weights_torch(K, N, workloads.seed_for("e0mx", "offline"), dev)
+    rows = []
+    for bits in (3, 5):
+        bpw = bits / 8.0 + 4.0 / 128.0
+        packed, scales = binding.tl_e0mx_quantize(w, bits)
+        ms = time_events(torch, lambda: binding.tl_e0mx_quantize(w, bits, packed=packed, scales=scales), 10)
+        row = {"bits": bits, "bytes_per_weight": bpw, "quantize_gbps": K * N * (4 + bpw) / (ms * 1e-3) / 1e9}
+        w_hat = binding.tl_e0mx_dequant(packed, scales, K, N, bits)
+        ms = time_events(torch, lambda: binding.tl_e0mx_dequant(packed, scales, K, N, bits, out=w_hat), 10)
+        row["dequant_gbps"] = K * N * (2 + bpw) / (ms * 1e-3) / 1e9
+        row["mae"] = float((w_hat.float() - w).abs().mean())
+        del w_hat
+        for M in (16, 2048):
+            x = workloads.activations_torch(M, K, workloads.seed_for("e0mx", "x", M), dev, 0.01 if M > 16 else 0.0)
+            y = torch.empty((M, N), dtype=torch.float16, device=dev)
+            ws = binding.tl_e0m4_workspace(max(256, int(binding.lib().tl_e0mx_matmul_workspace(M, K, N, bits))), dev)
+            run = lambda: binding.tl_e0mx_matmul(x, packed, scales, N, bits, y=y, workspace=ws)
+            for _ in range(3):
+                run()
+            us = time_events(torch, run, 10) * 1e3
+            row[f"matmul_m{M}"] = {"us": us, "gbps": (K * N * bpw + 2 * M * (K + N)) / us / 1e3,
+                                   "tflops": 2.0 * M * K * N / us / 1e6}
+        rows.append(row)
+    return rows
+
+
 def bench_list_sweep(binding, workloads, torch, dev, peaks, layers=4):
     """Batched decoding: `layers` ChatGLM2-6B-shaped layers (433 MB of weights at 4 layers, every matrix
     with its own activations) as ONE tl_e0m4_matmul_batch call against one tl_e0m4_matmul call per
@@ -988,6 +1019,7 @@ def run_native(args):
                    "sweep": lambda: bench_m_sweep(binding, workloads, torch, dev, peaks, args.stack, (args.M,),
                                                   layers=args.layers or 8),
                    "list_sweep": lambda: bench_list_sweep(binding, workloads, torch, dev, peaks),
+                   "e0mx": lambda: bench_e0mx(binding, workloads, torch, dev, peaks),
                    "chain": lambda: bench_decode_layer_chain(binding, workloads, torch, dev, peaks,
                                                              layers=args.layers or 6),
                    "prefill": lambda: bench_prefill(binding, workloads, torch, dev, peaks),
@@ -1114,24 +1146,30 @@ def run_native(args):
         del call_graph
         torch.cuda.empty_cache()
         if not args.no_prefill:
-            extra["prefill"] = bench_prefill(binding, workloads, torch, dev, peaks)
-            extra["quantize"], extra["dequant"] = bench_offline(binding, workloads, torch, dev)
-            extra["int4_twin"] = bench_int4_twin(binding, workloads, torch, dev, peaks)
-            extra["group_sizes"] = bench_group_sizes(binding, workloads, torch, dev, peaks)
-            extra["e0m8"] = bench_e0m8(binding, workloads, torch, dev, peaks)
-            extra["list_sweep"] = bench_list_sweep(binding, workloads, torch, dev, peaks)
+            def settled(fn, *a, **kw):
+                # every object starts from an idle GPU: the power-cap controller forgets the object before
+                torch.cuda.synchronize()
+                time.sleep(0.5)
+                return fn(*a, **kw)
+
+            extra["prefill"] = settled(bench_prefill, binding, workloads, torch, dev, peaks)
+            extra["quantize"], extra["dequant"] = settled(bench_offline, binding, workloads, torch, dev)
+            extra["int4_twin"] = settled(bench_int4_twin, binding, workloads, torch, dev, peaks)
+            extra["group_sizes"] = settled(bench_group_sizes, binding, workloads, torch, dev, peaks)
+            extra["e0m8"] = settled(bench_e0m8, binding, workloads, torch, dev, peaks)
+            extra["e0mx"] = settled(bench_e0mx, binding, workloads, torch, dev, peaks)
             extra["sweeps"] = {
-                "chatglm2_6b": bench_m_sweep(binding, workloads, torch, dev, peaks, "chatglm2_6b",
-                                             (1, 4, 16, 128, 512, 2048)),
-                "llm14b": bench_m_sweep(binding, workloads, torch, dev, peaks, "llm14b",
-                                        (1, 2, 4, 8, 16, 64, 256, 1024, 4096)),
+                "chatglm2_6b": settled(bench_m_sweep, binding, workloads, torch, dev, peaks, "chatglm2_6b",
+                                       (1, 4, 16, 128, 512, 2048)),
+                "llm14b": settled(bench_m_sweep, binding, workloads, torch, dev, peaks, "llm14b",
+                                  (1, 2, 4, 8, 16, 64, 256, 1024, 4096)),
             }
-            extra["launch_floor"] = bench_launch_floor(binding, torch, dev)
-            extra["decode_layer_chain"] = bench_decode_layer_chain(binding, workloads, torch, dev, peaks)
-            extra["rmsnorm"] = bench_rmsnorm(binding, workloads, torch, dev, peaks)
-            extra["matmul_add"] = bench_matmul_add(binding, workloads, torch, dev)
-            extra["matmul_swiglu"] = bench_matmul_swiglu(binding, workloads, torch, dev)
-            extra["kv_append"] = bench_kv_append(binding, workloads, torch, dev, peaks)
+            extra["launch_floor"] = settled(bench_launch_floor, binding, torch, dev)
+            extra["decode_layer_chain"] = settled(bench_decode_layer_chain, binding, workloads, torch, dev, peaks)
+            extra["rmsnorm"] = settled(bench_rmsnorm, binding, workloads, torch, dev, peaks)
+            extra["matmul_add"] = settled(bench_matmul_add, binding, workloads, torch, dev)
+            extra["matmul_swiglu"] = settled(bench_matmul_swiglu, binding, workloads, torch, dev)
+            extra["kv_append"] = settled(bench_kv_append, binding, workloads, torch, dev, peaks)
         if not args.no_cpu_baseline:
             cb_bytes, times, desc = time_oracle(args.stack, M, 3)
             extra["cpu_baseline"] = {"value": cb_bytes * len(times) / sum(times) / 1e9, "unit": UNIT,
@@ -1202,7 +1240,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = the stack's own)")
     ap.add_argument("--M", type=int, default=1)
     ap.add_argument("--object", default=None,
-                    choices=["e0m8", "sweep", "list_sweep", "chain", "prefill", "int4_twin", "launch_floor"],
+                    choices=["e0m8", "e0mx", "sweep", "list_sweep", "chain", "prefill", "int4_twin", "launch_floor"],
                     help="run only this extra object (at --M tokens where one applies) and print it")
     ap.add_argument("--no-prefill", action="store_true")
     ap.add_argument("--no-sustained", action="store_true")
