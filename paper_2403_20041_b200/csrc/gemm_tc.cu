@@ -26,7 +26,8 @@
 //   * warp 1    : one thread issues tcgen05.mma (M128 x N(tokens of the tile) x K16, A from tensor
 //                 memory, B from shared memory, fp32 accumulate) and commits each stage back to
 //                 both rings;
-//   * warps 19-22: epilogue.  tcgen05.ld gives a thread 32 tokens of one output column; the warp
+//   * warps 19-26: epilogue, two warps per tensor-memory lane quadrant taking the blocks of 32 tokens in
+//                 turn.  tcgen05.ld gives a thread 32 tokens of one output column; the warp
 //                 transposes 32 x 32 blocks through a small staging tile so that every thread
 //                 stores 16 bytes (eight neighbouring columns of a token), and it hands the
 //                 accumulator back as soon as the last block is in registers.  With split-K the
@@ -173,7 +174,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
       ptx::mbar_init(empty_p + 8 * s, BIG ? 4 : 8);  // the 4 warps of either half's stage read every chunk
     }
     ptx::mbar_init(acc_full, 1);
-    ptx::mbar_init(acc_empty, (PAIR ? 2 : 1) * kEpilogueWarps);
+    ptx::mbar_init(acc_empty, (PAIR ? 2 : 1) * kEpilogueWarpsTc);
     ptx::fence_mbar_init();
   }
   if (warp == 1) {
@@ -345,7 +346,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
   } else {
     // ------------------------------------------------------------------------- epilogue
     const int quad = warp & 3;          // the tensor-memory lane quadrant this warp may read
-    const int et = tid - (kFirstDequantWarp + kDequantWarps) * 32;  // 0..127 over the epilogue warps
+    const int et = tid - (kFirstDequantWarp + kDequantWarps) * 32;  // 0..255 over the epilogue warps
+    const int turn = (et >> 5) >> 2;    // which of the quadrant's two warps: it takes blocks turn, turn + 2, ...
     ptx::pdl_wait();
     int lt = 0;
     for (int item = unit; item < total_items && ok; item += units, ++lt) {
@@ -369,13 +371,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
         }
       };
       uint4 a_cur[4], a_nxt[4];
-      if constexpr (!SPLIT && ADD) load_add(a_cur, 0);
+      if constexpr (!SPLIT && ADD) load_add(a_cur, 32 * turn);
       if (!ptx::mbar_wait_bounded(acc_full, lt & 1, p.wait_limit)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t t_acc = tmem_base + ((uint32_t)(quad * 32) << 16);
       // Staging tile of this warp: [token 0..31][column 0..31] fp16, so that the global stores are
       // 16 bytes per thread (eight neighbouring columns of one token).
-      const uint32_t stg = smem0 + kOutStageOffset + (uint32_t)(et >> 5) * kOutStageBytes;
+      const uint32_t stg = smem0 + kOutStageOffsetTc + (uint32_t)(et >> 5) * kOutStageBytes;
       __half* y_chunk = p.y + (size_t)panel * 128 + quad * 32 + chunk * 8;
       // r[e] = this thread's output column at token mb + e: round, transpose through the staging
       // tile and store rows mb .. mb + 31 of the warp's 32 columns.
@@ -462,13 +464,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
       // consecutive bytes, which the L2 takes as one request.
       const int nl = quad * 32 + lane;
       float* tile_ws = SPLIT ? p.ws + (size_t)wi.tile * p.tok * 128 : nullptr;
+      // this warp's blocks of 32 tokens: turn, turn + 2, ... (the quadrant's other warp takes the rest);
+      // a warp without a block hands its share of the accumulator back at once
+      if (32 * turn >= rows_here) {
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (PAIR) mbar_arrive_cluster(acc_empty & kLeaderMask); else ptx::mbar_arrive(acc_empty);
+        }
+      }
 #pragma unroll 1
-      for (int mb = 0; mb < rows_here; mb += 32) {
+      for (int mb = 32 * turn; mb < rows_here; mb += 64) {
         uint32_t r[32];
         tmem_ld_32x32(t_acc + mb, r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (mb + 32 >= rows_here) {
-          // the accumulator is in registers: hand it back before the stores
+        if (mb + 64 >= rows_here) {
+          // this warp's last block is in registers: hand its share of the accumulator back before the stores
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           __syncwarp();
           if (lane == 0) {
@@ -477,7 +488,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
         }
         if constexpr (!SPLIT) {
           if constexpr (ADD) {
-            if (mb + 32 < rows_here) load_add(a_nxt, mb + 32);
+            if (mb + 64 < rows_here) load_add(a_nxt, mb + 64);
           }
           store_block(r, mb, a_cur);
           if constexpr (ADD) {
@@ -493,13 +504,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
       if constexpr (SPLIT) {
         // The CTA that arrives last at the tile converts the sums and leaves the scratch zero.
         __threadfence();
-        ptx::named_bar_sync(2, kEpilogueWarps * 32);
+        ptx::named_bar_sync(2, kEpilogueWarpsTc * 32);
         if (et == 0) {
           const unsigned prev = atomicAdd(p.cnt + wi.tile, 1u);
           asm volatile("st.shared.u32 [%0], %1;" ::"r"(last_flag), "r"(prev == (unsigned)p.ksplit - 1 ? 1u : 0u)
                        : "memory");
         }
-        ptx::named_bar_sync(2, kEpilogueWarps * 32);
+        ptx::named_bar_sync(2, kEpilogueWarpsTc * 32);
         uint32_t last;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(last) : "r"(last_flag) : "memory");
         if (last) {
@@ -509,7 +520,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
             float4* src = reinterpret_cast<float4*>(tile_ws);
             const int units = rows_here * 16;
 #pragma unroll 1
-            for (int unit = et; unit < units; unit += kEpilogueWarps * 32) {
+            for (int unit = et; unit < units; unit += kEpilogueWarpsTc * 32) {
               const int row = unit >> 4, b = (unit >> 1) & 7, h = unit & 1;
               const int q4 = row * 32 + 4 * b + h;          // float4 index of the gate quad
               const float4 g = __ldcg(src + q4), u = __ldcg(src + q4 + 2);
@@ -529,16 +540,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
             float4* src = reinterpret_cast<float4*>(tile_ws);
             const int n4 = rows_here * 32;
   #pragma unroll 1
-            for (int i0 = 0; i0 < n4; i0 += 4 * 128) {
+            for (int i0 = 0; i0 < n4; i0 += 4 * kEpilogueWarpsTc * 32) {
               float4 v[4];
   #pragma unroll
               for (int u = 0; u < 4; ++u) {
-                const int idx = i0 + u * 128 + et;
+                const int idx = i0 + u * kEpilogueWarpsTc * 32 + et;
                 v[u] = idx < n4 ? __ldcg(src + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
               }
   #pragma unroll
               for (int u = 0; u < 4; ++u) {
-                const int idx = i0 + u * 128 + et;
+                const int idx = i0 + u * kEpilogueWarpsTc * 32 + et;
                 if (idx < n4) {
                   const int m = m0 + (idx >> 5), c4 = (idx & 31) * 4;
                   __stcg(src + idx, make_float4(0.0f, 0.0f, 0.0f, 0.0f));
@@ -564,7 +575,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const TcParams p) {
           }
           if (et == 0) p.cnt[wi.tile] = 0;
         }
-        ptx::named_bar_sync(2, kEpilogueWarps * 32);
+        ptx::named_bar_sync(2, kEpilogueWarpsTc * 32);
       }
     }
   }
@@ -741,7 +752,7 @@ cudaError_t launch_gemm_tc(const __half* x, const uint32_t* packed, const uint32
   p.sx = kXRingBytes / round_bytes;
   if (p.sx > max_sx) p.sx = max_sx;
   if (bits == 8 && p.sx * round_bytes > 4 * 32768) --p.sx;  // the 16 KB slots need the room of a token box
-  p.pslots = (kOutStageOffset - p.sx * round_bytes) / tc_slot_bytes(bits, group);
+  p.pslots = (kOutStageOffsetTc - p.sx * round_bytes) / tc_slot_bytes(bits, group);
   if (p.pslots > kMaxPackedSlots) p.pslots = kMaxPackedSlots;
   if (p.pslots < 4) return cudaErrorInvalidConfiguration;  // the dequantizers' wait order relies on four slots
   p.ksplit = pl.ksplit;

@@ -32,8 +32,13 @@ constexpr int kBarOffset = kOutStageOffset + 4 * kOutStageBytes;
 constexpr int kSmemTotal = kBarOffset + 1024 + 1024;
 constexpr int kFirstDequantWarp = 3;
 constexpr int kDequantWarps = 16;         // 4 groups of 4 warps; a group covers the 128 lanes of a stage
-constexpr int kEpilogueWarps = 4;
-constexpr int kThreadsTc = (kFirstDequantWarp + kDequantWarps + kEpilogueWarps) * 32;
+constexpr int kEpilogueWarps = 4;         // list kernels: one warp per tensor-memory lane quadrant
+// The single-problem kernel drains its accumulator with TWO warps per lane quadrant, which take the
+// blocks of 32 tokens in turn: the accumulator goes back to the tensor core in half the time.  Its
+// eight staging tiles take the last packed slot's room.
+constexpr int kEpilogueWarpsTc = 8;
+constexpr int kOutStageOffsetTc = kOutStageOffset - (kEpilogueWarpsTc - kEpilogueWarps) * kOutStageBytes;
+constexpr int kThreadsTc = (kFirstDequantWarp + kDequantWarps + kEpilogueWarpsTc) * 32;
 constexpr int kAccCols = kTokTile;        // tensor-memory columns of the accumulator
 constexpr int kAStageCols = kStageK / 2;  // 32 columns: 64 fp16 per lane
 constexpr int kTmemCols = 512;            // 256 accumulator + 8 x 32 operand columns
