@@ -1137,7 +1137,9 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
         // ... and where all the clusters can be resident at once: a second wave would cost more
         // (asked for the largest shared-memory size a cluster launch uses: three stages at one token)
         const bool fits = panels <= lone_max_clusters(pow2, 128 + 3 * 36480 + smem_tail_cluster(1));
-        if (fits && (pow2 * 4 >= slices * 3 || tune(kTuneDecodeCluster) == 1)) {
+        // (or where a CTA's slice is a single ring stage anyway: then latency is all there is)
+        const bool one_stage = (p.prob[0].ng + pow2 - 1) / pow2 <= kStageGroups;
+        if (fits && (pow2 * 4 >= slices * 3 || one_stage || tune(kTuneDecodeCluster) == 1)) {
           slices = pow2;
           p.cluster = slices;
         }

@@ -57,3 +57,32 @@ def test_single_process_is_the_identity():
     assert replicas.max_over_ranks(3.5) == 3.5
     assert replicas.whole_job_throughput(4.0, 2.0, 1) == 2.0
     replicas.barrier(None)
+
+
+def test_bench_refuses_more_gpus_than_the_machine_has():
+    """`python bench.py --gpus N` outside a torchrun environment starts its own ranks; on a machine with
+    fewer GPUs it must fail loudly instead of running one replica and reporting n_gpus = 1."""
+    import subprocess
+    import sys
+
+    import torch
+
+    have = torch.cuda.device_count()
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", str(have + 2), "--steps", "1"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert res.returncode != 0
+    assert f"--gpus {have + 2}" in res.stderr and "CUDA device" in res.stderr
+    assert "n_gpus" not in res.stdout
+
+
+def test_bench_refuses_a_world_size_that_disagrees_with_gpus():
+    import subprocess
+    import sys
+
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "4", "--steps", "1"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert res.returncode != 0 and "WORLD_SIZE" in res.stderr
