@@ -1118,32 +1118,47 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
     // With fewer panels than CTAs every panel gets its own s CTAs, each taking one slice of the
     // panel's groups: a CTA then flushes one partial tile instead of the two of a range that
     // straddles a panel boundary, and with s = 1 none at all.  Measured at M = 1, 4, 8 on
-    // fourteen layer shapes, the largest s that fits is the fastest choice or within 3 % of it
-    // (up to 1.4x faster than the stream-K ranges), except that two slices of at most 8 groups
-    // lose to whole panels.
+    // fourteen layer shapes, slices are up to 1.4x faster than the stream-K ranges.
+    // The CTAs of a panel meet either in the global scratch (any s) or, launched as a cluster of s = 2,
+    // 4 or 8 neighbours, in one another's shared memory, which costs a fraction of the round trips
+    // (only where all clusters can be resident at once: a second wave would cost more than the
+    // exchange saves).  The choice minimises a small model fitted to per-launch times of sixteen
+    // layer shapes: ring stages a CTA walks (about 1 us each at this size) + 2.3 us for meeting in
+    // the scratch or 0.8 us for meeting in a cluster.
     int slices = 0;
+    bool cluster = false;
+    const int ng0 = p.prob[0].ng;
+    auto stages_of = [&](int s) { return (((ng0 + s - 1) / s) + kStageGroups - 1) / kStageGroups; };
     if (panels < grid && split_mode < 0 && forced_slices < 0) {
-      slices = grid / panels < p.prob[0].ng ? grid / panels : p.prob[0].ng;
-      if (slices == 2 && p.prob[0].ng <= 16) slices = 1;
-    }
-    if (forced_slices > 0 && split_mode < 0) slices = (int)forced_slices;
-    if (slices > 0 && slices <= p.prob[0].ng && (long long)panels * slices <= grid) {
-      // Two, four or eight CTAs per panel are launched as a cluster and add their partial sums up in
-      // shared memory, which costs a fraction of the round trips through the global scratch; other
-      // counts are rounded down to such a cluster (tl_e0m4_tuning_set("decode_cluster", 0) keeps them).
-      // (only where that keeps at least three quarters of the CTAs: seven slices stay seven).
-      if (NB == 1 && tune(kTuneDecodeCluster) != 0 && slices >= 2) {
-        const int pow2 = slices >= 8 ? 8 : (slices >= 4 ? 4 : 2);
-        // ... and where all the clusters can be resident at once: a second wave would cost more
-        // (asked for the largest shared-memory size a cluster launch uses: three stages at one token)
-        const bool fits = panels <= lone_max_clusters(pow2, 128 + 3 * 36480 + smem_tail_cluster(1));
-        // (or where a CTA's slice is a single ring stage anyway: then latency is all there is)
-        const bool one_stage = (p.prob[0].ng + pow2 - 1) / pow2 <= kStageGroups;
-        if (fits && (pow2 * 4 >= slices * 3 || one_stage || tune(kTuneDecodeCluster) == 1)) {
-          slices = pow2;
-          p.cluster = slices;
+      int nat = grid / panels < ng0 ? grid / panels : ng0;  // the most slices the grid allows
+      if (nat == 2 && ng0 <= 16) nat = 1;
+      slices = nat;
+      double best = stages_of(nat) + (nat > 1 ? 2.3 : 0.0);
+      if (nat > 1 && stages_of(1) <= best) {
+        slices = 1;
+        best = stages_of(1);
+      }
+      if (NB == 1 && tune(kTuneDecodeCluster) != 0) {
+        for (int c = 8; c >= 2; c >>= 1) {
+          if (c > ng0 || (long long)panels * c > grid) continue;
+          // (asked for the largest shared-memory size a cluster launch uses: three stages at one token)
+          if (panels > lone_max_clusters(c, 128 + 3 * 36480 + smem_tail_cluster(1))) continue;
+          const double cost = stages_of(c) + 0.8;
+          if (cost < best || (tune(kTuneDecodeCluster) == 1 && !cluster)) {
+            best = cost;
+            slices = c;
+            cluster = true;
+          }
         }
       }
+    }
+    if (forced_slices > 0 && split_mode < 0) {
+      slices = (int)forced_slices;
+      cluster = NB == 1 && tune(kTuneDecodeCluster) != 0 && (slices == 2 || slices == 4 || slices == 8) &&
+                panels <= lone_max_clusters(slices, 128 + 3 * 36480 + smem_tail_cluster(1));
+    }
+    if (slices > 0 && slices <= ng0 && (long long)panels * slices <= grid) {
+      if (cluster) p.cluster = slices;
       p.unit = -slices;
       grid = panels * slices;
     }
