@@ -333,7 +333,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
     }
     flags[0] = 0;
     if constexpr (PT::kCluster) {
-      if (p.cluster > 1) ptx::mbar_init(red_bar, kConsumerWarps);
+      if (p.cluster > 1) ptx::mbar_init(red_bar, 1);
     }
     ptx::fence_mbar_init();
   }
@@ -822,21 +822,28 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
             const uint32_t base = ptx::cluster_ctarank() - (uint32_t)my_i;     // cluster rank of the group's first CTA
             const uint32_t dst = base + (uint32_t)(warp % s_grp);              // who finishes this warp's tile
             const int per = kPanelTiles / s_grp;                               // tiles every CTA finishes
+            // The receiver announces what it expects: s contributions of 16 columns x M tokens for each
+            // of its tiles that exist (the byte count may be reported before or after it is announced).
+            if (tid == 0) {
+              int mine_tiles = 0;
+              for (int u = 0; u < per; ++u) mine_tiles += (u * s_grp + my_i < R) ? 1 : 0;
+              ptx::mbar_arrive_expect_tx(red_bar, (uint32_t)(mine_tiles * s_grp * kTileN * M * 4));
+            }
             if (warp < R) {
               constexpr int kRedPad = 8 * MT;
               const uint32_t to = ptx::mapa(red_buf + (uint32_t)((my_i * per + warp / s_grp) * kTileN * kRedPad * 4), dst);
+              const uint32_t to_bar = ptx::mapa(red_bar, dst);
 #pragma unroll
               for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                   const int m = 8 * mt + 2 * t + (j & 1);
-                  if (m < M) ptx::st_cluster_f32(to + (uint32_t)(((gid + (j >> 1) * 8) * kRedPad + m) * 4), acc[mt][j]);
+                  if (m < M)
+                    ptx::st_async_cluster_f32(to + (uint32_t)(((gid + (j >> 1) * 8) * kRedPad + m) * 4), acc[mt][j], to_bar);
                 }
               }
             }
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_release_cluster(ptx::mapa(red_bar, dst));
-            // all eight warps of all s CTAs have arrived here once the phase completes
+            // every contribution has landed once the phase completes
             if (!ptx::mbar_wait_bounded_cluster(red_bar, red_phase, p.wait_limit)) {
               if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
               return;

@@ -98,6 +98,14 @@ __device__ __forceinline__ uint32_t mapa(uint32_t smem_addr, uint32_t rank) {
 __device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
 }
+// A store into another CTA's shared memory that reports its four bytes to a barrier of that CTA when
+// it has landed: the receiver that sees the barrier's phase complete sees the data, and the sender
+// needs neither a fence nor an arrival of its own.
+__device__ __forceinline__ void st_async_cluster_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(cluster_addr),
+               "r"(__float_as_uint(v)), "r"(cluster_bar)
+               : "memory");
+}
 // Arrive on a barrier of another CTA of the cluster; what this thread (and, through a preceding
 // __syncwarp, its warp) wrote before becomes visible to the thread that acquires the phase.
 __device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_bar) {
