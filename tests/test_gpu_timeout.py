@@ -96,3 +96,30 @@ def test_wait_runs_out_in_the_list_kernels(lib, dev, tuning, M):
     for (_, _, _, y_ref), y in zip(cases, ys):
         _check(y, y_ref)
     assert lib.tl_e0m4_device_status() == 0
+
+
+def test_wait_runs_out_in_the_chain_kernel(lib, dev, tuning):
+    # two dependent steps; with the producers silent every consumer gives up on its first stage, the
+    # kernel returns, and the re-initialised workspace (scratch slots and phase counters) serves a normal call
+    M, K, N = 2, 256, 256
+    x, p1, s1, ref1 = _case(lib, dev, M, K, N, seed=71)
+    w2 = workloads.weights(N, 128, 72)
+    p2, s2 = lib.tl_e0m4_quantize(torch.from_numpy(w2).to(dev))
+    t = torch.zeros((M, N), dtype=torch.float16, device=dev)
+    y = torch.zeros((M, 128), dtype=torch.float16, device=dev)
+    steps = [dict(x=x, packed=p1, scales=s1, y=t), dict(x=t, packed=p2, scales=s2, y=y, after_previous=True)]
+    ws = lib.tl_e0m4_workspace(lib.tl_e0m4_matmul_chain_workspace(), dev)
+    tuning("wait_limit_cycles", SHORT)
+    tuning("skip_copies", 1)
+    lib.tl_e0m4_matmul_chain(steps, M, ws)
+    assert lib.tl_e0m4_device_status() == TL_ERR_TIMEOUT
+    tuning("skip_copies", -1)
+    tuning("wait_limit_cycles", -1)
+    lib.lib().tl_e0m4_workspace_init(ws.data_ptr(), ws.numel(), None)
+    lib.tl_e0m4_matmul_chain(steps, M, ws)
+    torch.cuda.synchronize()
+    _check(t, ref1)
+    codes, d_h, b_h = oracle.quantize(w2)
+    _check(y, oracle.matmul(t.cpu().numpy(), oracle.dequantize(codes, d_h, b_h)))
+    assert lib.tl_e0m4_device_status() == 0
+    assert not ws.cpu().numpy().any()
