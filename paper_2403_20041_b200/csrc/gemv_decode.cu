@@ -53,6 +53,9 @@ __host__ __device__ constexpr int x_offset(int group) { return kScaleOffset + kS
 constexpr int kXRowBytes = kStageGroups * 256 + 32;
 constexpr int kWsPad = 16;                           // scratch floats per output column
 constexpr int kMaxStages = 4;
+// the 64 zero bytes that stand in for missing token rows follow the barriers and two flag words and
+// are read with 16-byte loads
+static_assert((3 * kMaxStages * 8 + 16) % 16 == 0, "an odd number of ring stages would misalign the zero block");
 
 // Panels whose k groups are shared by the s = 2, 4 or 8 CTAs of (a part of) a cluster meet in
 // shared memory instead of the global scratch: every CTA sends the partial sums of tile t to the
