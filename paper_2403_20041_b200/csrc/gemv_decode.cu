@@ -225,6 +225,59 @@ constexpr uint32_t kMaskLo = 0x000F000Fu, kExpLo = 0x58005800u;  // 128 + code/8
 constexpr uint32_t kMaskHi = 0x00F000F0u, kExpHi = 0x48004800u;  // 8 + code/8
 constexpr float kOffLo = 126.0f, kOffHi = 6.0f;
 
+// Row sums of one ring stage on the tensor core (the row-sum warp).  Both numbers the consumers
+// need per token and group come out of one product with the activations as the 16-row operand:
+// against a column of ones the plain sum (it multiplies the bias), against a column of -126 / -6
+// minus the total of the constant offsets (it seeds the consumers' accumulator).  A lane's 16
+// bytes are eight consecutive k: the halves 0,1 and 4,5 (k % 4 < 2, offset 126) become the first
+// eight k of a product, the halves 2,3 and 6,7 (offset 6) its last eight; the order of k inside
+// a sum does not matter.
+// The 16 rows are filled whatever the token count T (2, 4, 8 or 16 tokens per row set): row r is
+// token r % T, and r / T counts through the groups of the stage; with two tokens the eight rows
+// left over take the second half of each group's k, and a lane adds the two halves up.  All
+// chains run without a branch; a group the stage does not have reads stale bytes of the stage's
+// own activation rows and is not stored.  b_first / b_last: the constant operand of this lane.
+template <int T>
+__device__ __forceinline__ void stage_row_sums(uint32_t x_rows, float* xsum, int M, int groups, int lane,
+                                               uint32_t b_first, uint32_t b_last) {
+  constexpr int kSets = T * kStageGroups > 16 ? T * kStageGroups / 16 : 1;  // products side by side: 1, 1, 2, 4
+  constexpr int kGroupsPerSet = kStageGroups / kSets;
+  constexpr bool kHalves = T * kStageGroups < 16;  // T = 2: rows 8..15 are the second half of k
+  constexpr int kChunks = kHalves ? 2 : 4;         // 64-byte pieces of k per row
+  const int gid = lane >> 2, t = lane & 3;
+  // rows gid and gid + 8: token, group inside the set, half of k
+  const int m_lo = gid % T, i_lo = gid / T, m_hi = (gid + 8) % T, i_hi = (gid + 8) / T;
+  const int g_lo = i_lo % kGroupsPerSet, g_hi = i_hi % kGroupsPerSet;
+  const bool has_lo = m_lo < M, has_hi = m_hi < M;
+  const uint32_t at_lo = x_rows + m_lo * kXRowBytes + g_lo * 256 + (i_lo / kGroupsPerSet) * 128 + t * 16;
+  const uint32_t at_hi = x_rows + m_hi * kXRowBytes + g_hi * 256 + (i_hi / kGroupsPerSet) * 128 + t * 16;
+  float c[kSets][2][4];
+#pragma unroll
+  for (int rs = 0; rs < kSets; ++rs) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[rs][0][i] = c[rs][1][i] = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kChunks; ++j) {
+      const uint32_t off = rs * kGroupsPerSet * 256 + j * 64;
+      const uint4 lo = has_lo ? ptx::lds128(at_lo + off) : make_uint4(0u, 0u, 0u, 0u);
+      const uint4 hi = has_hi ? ptx::lds128(at_hi + off) : make_uint4(0u, 0u, 0u, 0u);
+      mma16816(c[rs][0], lo.x, hi.x, lo.y, hi.y, b_first, b_last);
+      mma16816(c[rs][1], lo.z, hi.z, lo.w, hi.w, b_first, b_last);
+    }
+  }
+  if (t == 0) {
+#pragma unroll
+    for (int rs = 0; rs < kSets; ++rs) {
+      float2 lo = make_float2(c[rs][0][0] + c[rs][1][0], c[rs][0][1] + c[rs][1][1]);
+      const float2 hi = make_float2(c[rs][0][2] + c[rs][1][2], c[rs][0][3] + c[rs][1][3]);
+      if (kHalves) lo = make_float2(lo.x + hi.x, lo.y + hi.y);
+      const int gl = rs * kGroupsPerSet + g_lo, gh = rs * kGroupsPerSet + g_hi;
+      if (gl < groups && has_lo) *reinterpret_cast<float2*>(xsum + (gl * 16 + m_lo) * 2) = lo;
+      if (!kHalves && gh < groups && has_hi) *reinterpret_cast<float2*>(xsum + (gh * 16 + m_hi) * 2) = hi;
+    }
+  }
+}
+
 // Walks the CTA's chunk range stage by stage, across problems: a stage never crosses a panel end.
 // For a chain the walk goes on through the phases: when the CTA's range of one phase is used up it
 // moves to the CTA's range of the next phase in which it has any chunks.
@@ -477,8 +530,12 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
     // ------------------------------------------------- row sums of the activation slices
     ptx::pdl_wait();
     int s = 0, phase = 0;
-    static_assert(kStageGroups == 4, "the row-sum warp gives 8 lanes to each group of a stage");
-    const int sub = lane >> 3, part = lane & 7;  // group of the stage, 16-halves slice of its 128 k
+    // the constant operand of the row-sum products: even columns all ones, odd columns minus the
+    // offset of the k's class
+    const int gid = lane >> 2;
+    const __half2 neg_lo = __float2half2_rn(-kOffLo), neg_hi = __float2half2_rn(-kOffHi);
+    const uint32_t b_first = (gid & 1) ? *reinterpret_cast<const uint32_t*>(&neg_lo) : 0x3C003C00u;
+    const uint32_t b_last = (gid & 1) ? *reinterpret_cast<const uint32_t*>(&neg_hi) : 0x3C003C00u;
     const uint32_t ring_h = ptx::smem_u32(ring);
     [[maybe_unused]] int rms_last = -1;  // chain: the step whose row factors were formed last
     for (StageWalk<PT> w = make_walk(); !w.done(); w.next()) {
@@ -488,33 +545,18 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
       }
       const uint32_t st = ring_h + s * p.stage_bytes;
       float* xsum = reinterpret_cast<float*>(ring + (size_t)s * p.stage_bytes + p.xsum_offset);
-      const bool live = sub < w.groups();
-      for (int m = 0; G == kGroup && m < M; ++m) {  // smaller groups need no sums
-        // sum_a: the k with k % 4 < 2 (they carry the offset 126), sum_b: the others (offset 6)
-        float sum_a = 0.0f, sum_b = 0.0f;
-        if (live) {
-          const uint32_t row = st + kXOffset + m * kXRowBytes + sub * 256 + part * 16;
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const uint4 v = ptx::lds128(row + j * 128);
-            const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
-            const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
-            const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&v.z));
-            const float2 f3 = __half22float2(*reinterpret_cast<const __half2*>(&v.w));
-            sum_a += (f0.x + f0.y) + (f2.x + f2.y);
-            sum_b += (f1.x + f1.y) + (f3.x + f3.y);
-          }
+      if constexpr (G == kGroup) {  // smaller groups need no sums
+        const uint32_t x_rows = st + kXOffset;
+        const int groups = w.groups();
+        if constexpr (MT == 2) {
+          stage_row_sums<16>(x_rows, xsum, M, groups, lane, b_first, b_last);
+        } else if (M <= 2) {
+          stage_row_sums<2>(x_rows, xsum, M, groups, lane, b_first, b_last);
+        } else if (M <= 4) {
+          stage_row_sums<4>(x_rows, xsum, M, groups, lane, b_first, b_last);
+        } else {
+          stage_row_sums<8>(x_rows, xsum, M, groups, lane, b_first, b_last);
         }
-#pragma unroll
-        for (int off = 1; off < 8; off <<= 1) {
-          sum_a += __shfl_xor_sync(0xFFFFFFFFu, sum_a, off);
-          sum_b += __shfl_xor_sync(0xFFFFFFFFu, sum_b, off);
-        }
-        // what the consumers need: the plain sum (times the bias) and the total of the constant
-        // offsets, negated so that it can seed the tensor-core accumulator
-        if (live && part == 0)
-          *reinterpret_cast<float2*>(xsum + (sub * 16 + m) * 2) =
-              make_float2(sum_a + sum_b, -(kOffLo * sum_a + kOffHi * sum_b));
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(full0 + 8 * s);
