@@ -744,11 +744,10 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
             for (int mt = 0; mt < MT; ++mt) {
               if (v == 0) {
                 mma16816_init(c[mt][0], l01, h01, l23, h23, xv[mt][v].x, xv[mt][v].y, xs[mt].y, xs[mt].w);
-                mma16816_init(c[mt][1], l45, h45, l67, h67, xv[mt][v].z, xv[mt][v].w, 0.0f, 0.0f);
               } else {
                 mma16816(c[mt][0], l01, h01, l23, h23, xv[mt][v].x, xv[mt][v].y);
-                mma16816(c[mt][1], l45, h45, l67, h67, xv[mt][v].z, xv[mt][v].w);
               }
+              mma16816(c[mt][0], l45, h45, l67, h67, xv[mt][v].z, xv[mt][v].w);
             }
           }
 
@@ -756,10 +755,10 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           const float2 db_hi = __half22float2(*reinterpret_cast<const __half2*>(&s_hi));
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
-            const float t0 = fmaf(-db_lo.y, xs[mt].x, c[mt][0][0] + c[mt][1][0]);
-            const float t1 = fmaf(-db_lo.y, xs[mt].z, c[mt][0][1] + c[mt][1][1]);
-            const float t2 = fmaf(-db_hi.y, xs[mt].x, c[mt][0][2] + c[mt][1][2]);
-            const float t3 = fmaf(-db_hi.y, xs[mt].z, c[mt][0][3] + c[mt][1][3]);
+            const float t0 = fmaf(-db_lo.y, xs[mt].x, c[mt][0][0]);
+            const float t1 = fmaf(-db_lo.y, xs[mt].z, c[mt][0][1]);
+            const float t2 = fmaf(-db_hi.y, xs[mt].x, c[mt][0][2]);
+            const float t3 = fmaf(-db_hi.y, xs[mt].z, c[mt][0][3]);
             acc[mt][0] = fmaf(db_lo.x, t0, acc[mt][0]);
             acc[mt][1] = fmaf(db_lo.x, t1, acc[mt][1]);
             acc[mt][2] = fmaf(db_hi.x, t2, acc[mt][2]);
