@@ -40,7 +40,7 @@ if ROOT not in sys.path:
 # figure was captured on 8 of the 40 layers (a capture has to stay small) and is scaled by the layer
 # count: a launch's traffic is its weights, read once, so it grows in proportion.  Other workloads
 # report null.
-DECODE_TRAFFIC_BYTES_PER_LAYER_M1 = {"gemma2b": (1.0598e9 + 7.0e6) / 18, "llm14b": (1.342895e9 + 4.67e6) / 8}
+DECODE_TRAFFIC_BYTES_PER_LAYER_M1 = {"gemma2b": (1.05985e9 + 6.27e6) / 18, "llm14b": (1.343138e9 + 5.04e6) / 8}
 
 METRIC = "e0m4_decode_gemv_hbm_gbps"
 UNIT = "GB/s"
