@@ -646,6 +646,15 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
   for (int v = 0; v < 4; ++v) chunk_off[v] = ((v + (rot ? 1 : 0)) & 3) * 16;
   const uint32_t ring_u32 = ptx::smem_u32(ring);
 
+  [[maybe_unused]] auto addend = [&](const auto& q, int m, size_t n) -> float {
+    if constexpr (CHAIN) return __half2float(__ldcg(q.add + (size_t)m * q.add_stride + n));  // L2: other SMs wrote it
+    else return __half2float(p.add[(size_t)m * p.add_stride + n]);
+  };
+  [[maybe_unused]] float add_pre[MT][4];  // addend of the outputs this lane emits at the end of the current panel
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) add_pre[mt][j] = 0.0f;
   StageWalk<PT> w = make_walk();
   [[maybe_unused]] uint32_t red_phase = 0;  // cluster launches: parity of the next exchange
   int g_begin = w.g;
@@ -658,6 +667,37 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
     if (!ptx::mbar_wait_bounded(full0 + 8 * s, phase, p.wait_limit)) {
       if (lane == 0) atomicExch(p.status, (unsigned)TL_ERR_TIMEOUT);
       return;  // every wait in this kernel is bounded, so the other warps leave as well
+    }
+    // The stage that ends the panel (or the range): the addend of the outputs this lane will emit
+    // is requested now, so that its trip to L2 runs under the stage's products instead of after them.
+    if constexpr (CHAIN || EPI == 1) {
+      const bool ends = (w.g + groups == w.ng) || (w.left - groups <= 0);
+      int epi_now = EPI;
+      if constexpr (CHAIN) epi_now = q.epi;
+      if (ends && epi_now == 1) {
+        int tile = warp;         // the tile whose outputs this warp stores
+        bool mine = warp < R;
+        if constexpr (PT::kCluster) {
+          const bool whole = g_begin == 0 && w.g + groups == w.ng;
+          int unit;
+          if constexpr (CHAIN) unit = p.phase[w.ph].unit; else unit = p.unit;
+          if (!whole && unit < 0 && p.cluster > 1) {  // shared inside a cluster: see the exchange below
+            const int s_grp = -unit, s_log = 31 - __clz(s_grp);
+            tile = warp * s_grp + (int)(blockIdx.x & (unsigned)(s_grp - 1));
+            mine = warp < (kPanelTiles >> s_log) && tile < R;
+          }
+        }
+        if (mine) {
+          const size_t n0 = (size_t)(w.panel * kPanelTiles + tile) * kTileN + gid;
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int m = 8 * mt + 2 * t + (j & 1);
+              if (m < M) add_pre[mt][j] = addend(q, m, n0 + (j >> 1) * 8);
+            }
+        }
+      }
     }
     if (warp < R) {
       const uint32_t st = ring_u32 + s * p.stage_bytes;
@@ -810,12 +850,8 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           r_odd = rms_val[slot * 8 + 2 * t + 1];
         }
       }
-      auto addend = [&](int m, size_t n) -> float {
-        if constexpr (CHAIN) return __half2float(__ldcg(q.add + (size_t)m * q.add_stride + n));  // L2: other SMs wrote it
-        else return __half2float(p.add[(size_t)m * p.add_stride + n]);
-      };
       // one finished output (and, for SwiGLU, its partner 8 columns on): the epilogue and the store
-      auto emit = [&](int m, size_t n, float v, float v_up, int j) {
+      auto emit = [&](int m, size_t n, float v, float v_up, int j, int mt) {
         if (CHAIN) {
           const float r = (j & 1) ? r_odd : r_even;
           v *= r;
@@ -826,7 +862,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           // outputs silu(gate) * up go to columns 8 * tile + gid of y[M, N / 2]
           if (j < 2) q.y[(size_t)m * (q.N >> 1) + (n - gid) / 2 + gid] = __float2half_rn(swiglu(v, v_up));
         } else {
-          if (epi == 1) v += addend(m, n);
+          if (epi == 1) v += add_pre[mt][j];
           q.y[(size_t)m * q.N + n] = __float2half_rn(v);
         }
       };
@@ -839,7 +875,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int m = 8 * mt + 2 * t + (j & 1);
-              if (m < M) emit(m, n_lo + (j >> 1) * 8, acc[mt][j], acc[mt][(j + 2) & 3], j);
+              if (m < M) emit(m, n_lo + (j >> 1) * 8, acc[mt][j], acc[mt][(j + 2) & 3], j, mt);
             }
           }
         }
@@ -861,11 +897,12 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
           if (unit < 0 && p.cluster > 1) {
             // ---- the s CTAs that share this panel are neighbours in a cluster: exchange through shared memory
             exchanged = true;
-            const int s_grp = -unit;
-            const int my_i = (int)(blockIdx.x % (unsigned)s_grp);               // slice of the panel = rank in the group
+            const int s_grp = -unit;                                           // 2, 4 or 8
+            const int s_log = 31 - __clz(s_grp);
+            const int my_i = (int)(blockIdx.x & (unsigned)(s_grp - 1));         // slice of the panel = rank in the group
             const uint32_t base = ptx::cluster_ctarank() - (uint32_t)my_i;     // cluster rank of the group's first CTA
-            const uint32_t dst = base + (uint32_t)(warp % s_grp);              // who finishes this warp's tile
-            const int per = kPanelTiles / s_grp;                               // tiles every CTA finishes
+            const uint32_t dst = base + (uint32_t)(warp & (s_grp - 1));        // who finishes this warp's tile
+            const int per = kPanelTiles >> s_log;                              // tiles every CTA finishes
             // The receiver announces what it expects: s contributions of 16 columns x M tokens for each
             // of its tiles that exist (the byte count may be reported before or after it is announced).
             if (tid == 0) {
@@ -875,7 +912,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
             }
             if (warp < R) {
               constexpr int kRedPad = 8 * MT;
-              const uint32_t to = ptx::mapa(red_buf + (uint32_t)((my_i * per + warp / s_grp) * kTileN * kRedPad * 4), dst);
+              const uint32_t to = ptx::mapa(red_buf + (uint32_t)((my_i * per + (warp >> s_log)) * kTileN * kRedPad * 4), dst);
               const uint32_t to_bar = ptx::mapa(red_bar, dst);
 #pragma unroll
               for (int mt = 0; mt < MT; ++mt) {
@@ -921,11 +958,11 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                   const int m = 8 * mt + 2 * t + (j & 1);
-                  if (m < M) emit(m, n_out + (j >> 1) * 8, v[j], v[(j + 2) & 3], j);
+                  if (m < M) emit(m, n_out + (j >> 1) * 8, v[j], v[(j + 2) & 3], j, mt);
                 }
               }
             }
-            final_share = kPanelTiles / s_grp;
+            final_share = per;
           }
         }
         int k = panel;
@@ -970,7 +1007,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
                   // SwiGLU: the up half (j >= 2) is read by the iteration of its gate and cleared by its own
                   const float v = __ldcg(a);
                   const float v_up = (epi == 2 && j < 2) ? __ldcg(a + 8 * kWsPad) : 0.0f;
-                  emit(m, n_lo + (j >> 1) * 8, v, v_up, j);
+                  emit(m, n_lo + (j >> 1) * 8, v, v_up, j, mt);
                   __stcg(a, 0.0f);
                 }
               }
