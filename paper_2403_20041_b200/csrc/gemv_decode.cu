@@ -5,13 +5,15 @@
 //   * The packed stream is a sequence of chunks: chunk (panel p, group g) holds the tiles of up
 //     to 8 neighbouring column blocks (128 columns) for one 128-k group, 8 KB of codes plus
 //     512 B of scale words, contiguous in memory; consecutive g follow each other.  The chunk
-//     sequence is cut into equal contiguous ranges, one per CTA (at most one CTA per SM),
+//     sequence is cut into equal contiguous ranges, one per CTA (at most two CTAs per SM),
 //     either on panel boundaries or, when that would leave SMs idle, anywhere ("stream-K").
 //   * A stage of the shared-memory ring holds up to kStageGroups consecutive chunks of one
 //     panel.  Warp 8 is the producer: one thread fills the ring with bulk asynchronous copies
 //     (TMA) that complete on mbarriers: codes, scale words and the matching slice of every
-//     activation row.  Warp 9 adds up each activation row per group (sum_k x) for the
-//     consumers as soon as the slice has landed.
+//     activation row.  Warp 9 adds up each activation row per group (sum_k x, and the total of
+//     the binade offsets) as soon as the slice has landed, with one tensor-core product per 32 k
+//     against a constant operand (stage_row_sums), and only then hands the stage to the
+//     consumers: its time per stage is latency on the ring's critical path.
 //   * Warps 0-7 are consumers; warp r owns column block r of the panel and keeps its fp32
 //     accumulators in registers over all groups.  Per tile a lane reads 2 x 16 bytes of
 //     codes, rebuilds the fp16 numbers 2 + code/8 with the shift/mask/OR of Section 2.3 and
