@@ -146,3 +146,36 @@ def test_chain_of_random_steps(lib, dev, case):
         addend = _np(st["addend"]) if "addend" in st else None
         ref = oracle.chain_step(_np(st["x"]), w_hat, epi, addend, st.get("rms_eps"))
         assert_close(_np(st["y"]), ref)
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_single_call_at_prefill_sizes(lib, dev, case):
+    """41..700 tokens: the tensor-core kernel's token tiles, split-K, pairs of CTAs and rounds of a
+    group, on shapes with ragged panels and ragged token tiles, with every epilogue."""
+    rng = np.random.default_rng(workloads.seed_for("random prefill", case))
+    _, K, N, group = _draw(rng)
+    M = int(rng.integers(41, 701))
+    epi = ["none", "add", "bias", "swiglu"][case % 4]
+    w_np = workloads.weights(K, N, workloads.seed_for("random prefill w", case))
+    x_np = workloads.activations(M, K, workloads.seed_for("random prefill x", case), outlier_fraction=0.01)
+    packed, scales = lib.tl_e0m4_quantize(torch.from_numpy(w_np).to(dev), group=group)
+    x = torch.from_numpy(x_np).to(dev)
+    w_hat = _w_hat(w_np, group)
+    if epi == "none":
+        y = lib.tl_e0m4_matmul(x, packed, scales, N, group=group)
+        ref = oracle.matmul(x_np, w_hat)
+    elif epi == "add":
+        a_np = workloads.activations(M, N, workloads.seed_for("random prefill a", case))
+        y = lib.tl_e0m4_matmul_add(x, packed, scales, N, torch.from_numpy(a_np).to(dev),
+                                   y=torch.empty((M, N), dtype=torch.float16, device=dev), group=group)
+        ref = oracle.matmul(x_np, w_hat, a_np)
+    elif epi == "bias":
+        b_np = workloads.activations(1, N, workloads.seed_for("random prefill b", case))[0].copy()
+        y = lib.tl_e0m4_matmul_bias(x, packed, scales, N, torch.from_numpy(b_np).to(dev), group=group)
+        ref = oracle.matmul(x_np, w_hat, b_np)
+    else:
+        y = lib.tl_e0m4_matmul_swiglu(x, packed, scales, N, group=group)
+        ref = oracle.swiglu_blocks(oracle.matmul(x_np, w_hat))
+    torch.cuda.synchronize()
+    assert lib.tl_e0m4_device_status() == 0
+    assert_close(_np(y), ref)
