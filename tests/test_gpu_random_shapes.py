@@ -179,3 +179,30 @@ def test_single_call_at_prefill_sizes(lib, dev, case):
     torch.cuda.synchronize()
     assert lib.tl_e0m4_device_status() == 0
     assert_close(_np(y), ref)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_other_code_widths_on_random_shapes(lib, dev, case):
+    """E0M8, E0M3 and E0M5 (groups of 128): quantizer words bit for bit and the matmul within
+    tolerance, 1..300 tokens, shapes drawn like the 4-bit cases."""
+    rng = np.random.default_rng(workloads.seed_for("random widths", case))
+    _, K, N, _ = _draw(rng)
+    group = 128
+    M = int(rng.choice([1, 2, 5, 8, 9, 16, int(rng.integers(17, 301))]))
+    bits = [8, 3, 5][case % 3]
+    w_np = workloads.weights(K, N, workloads.seed_for("random widths w", case))
+    x_np = workloads.activations(M, K, workloads.seed_for("random widths x", case))
+    w, x = torch.from_numpy(w_np).to(dev), torch.from_numpy(x_np).to(dev)
+    codes, d_h, b_h = oracle.quantize(w_np, group=group, bits=bits)
+    ref_p, ref_s = oracle.pack(codes, d_h, b_h, group=group, bits=bits)
+    if bits == 8:
+        packed, scales = lib.tl_e0m8_quantize(w, group=group)
+        y = lib.tl_e0m8_matmul(x, packed, scales, N, group=group)
+    else:
+        packed, scales = lib.tl_e0mx_quantize(w, bits)
+        y = lib.tl_e0mx_matmul(x, packed, scales, N, bits)
+    torch.cuda.synchronize()
+    assert lib.tl_e0m4_device_status() == 0
+    assert np.array_equal(_np(packed).view(np.uint32), ref_p)
+    assert np.array_equal(_np(scales).view(np.uint32), ref_s)
+    assert_close(_np(y), oracle.matmul(x_np, oracle.dequantize(codes, d_h, b_h, group=group, bits=bits)))
