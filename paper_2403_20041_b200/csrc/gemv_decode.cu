@@ -1262,8 +1262,9 @@ cudaError_t launch_batch(const DecodeProblem* probs, int count, int M, void* wor
   stages = stages > kMaxStages ? kMaxStages : (stages < 2 ? 2 : stages);
   p.stages = stages;
   const size_t smem = 128 + (size_t)stages * p.stage_bytes + 3 * kMaxStages * sizeof(uint64_t) + 16 + 64;
-  // measured crossover: below five tokens the selects cost more than the conflicts they avoid
-  const int rot_min = tune(kTuneDecodeRotMin) >= 0 ? (int)tune(kTuneDecodeRotMin) : 5;
+  // measured crossover: below five tokens the selects cost more than the conflicts they avoid; a
+  // list (bound by its consumers' issue slots, not by latency) gains only from seven tokens on
+  const int rot_min = tune(kTuneDecodeRotMin) >= 0 ? (int)tune(kTuneDecodeRotMin) : (NB == 1 ? 5 : 7);
   cudaError_t e;
   if constexpr (NB == 1) {
     if (p.add) {
