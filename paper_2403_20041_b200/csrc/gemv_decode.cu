@@ -398,17 +398,28 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
   if (tid < 16) reinterpret_cast<uint32_t*>(bars + 3 * kMaxStages + 2)[tid] = 0u;
   if (CHAIN && tid < kChainRmsSlots) rms_step[tid] = -1;
   __syncthreads();
+  // Every CTA's exchange barrier has to exist before a neighbour arrives on it.  All threads arrive
+  // at the cluster barrier here and wait for it where they would be idle anyway (cluster_ready):
+  // the producer after it has requested its first stages, everybody else at once.
+  [[maybe_unused]] const bool clustered = PT::kCluster && p.cluster > 1;
   if constexpr (PT::kCluster) {
-    // every CTA's exchange barrier exists before a neighbour arrives on it (all threads are still here)
-    if (p.cluster > 1) ptx::cluster_sync_all();
+    if (clustered) ptx::cluster_arrive_release();
   }
+  auto cluster_ready = [&]() {
+    if constexpr (PT::kCluster) {
+      if (clustered) ptx::cluster_wait_acquire();
+    }
+  };
   ptx::pdl_launch_dependents();
 
   // this CTA's contiguous range of chunks (a chain has one per phase: see StageWalk)
   int c0 = 0, c1 = 0;
   if constexpr (!CHAIN) {
     cta_range(p.total_chunks, p.unit, p.prob[0].ng, p.prob[0].panels, c0, c1);
-    if (c1 <= c0) return;
+    if (c1 <= c0) {
+      cluster_ready();
+      return;
+    }
   }
   const int n_chunks = c1 - c0;
   const int M = p.M;
@@ -419,7 +430,10 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------------- producer
-    if (lane != 0 || p.skip_copies) return;
+    if (lane != 0 || p.skip_copies) {
+      cluster_ready();
+      return;
+    }
     const uint32_t ring_s = ptx::smem_u32(ring);
     auto issue_w = [&](const StageWalk<PT>& w, int s) {
       const auto& q = p.prob[w.j];
@@ -451,6 +465,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
       // earlier phase is complete (the counter of final panels has reached the phase's target),
       // because the slice is some earlier step's output.  Neither cursor blocks the other: both
       // conditions are probed without waiting.
+      cluster_ready();
       StageWalk<PT> w = make_walk();
       StageWalk<PT> wx = w;
       int iw = 0, ix = 0;            // stages whose weights / activations have been requested
@@ -505,6 +520,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
       issue_w(w, issued);
       w.next();
     }
+    cluster_ready();
     ptx::pdl_wait();
     for (int i = 0; i < issued; ++i) {
       issue_x(wx, i);
@@ -530,6 +546,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
 
   if (warp == kConsumerWarps + 1) {
     // ------------------------------------------------- row sums of the activation slices
+    cluster_ready();
     ptx::pdl_wait();
     int s = 0, phase = 0;
     // the constant operand of the row-sum products: even columns all ones, odd columns minus the
@@ -615,6 +632,7 @@ gemv_decode_kernel(const __grid_constant__ PT p) {
   }
 
   // ---------------------------------------------------------------------- consumers
+  cluster_ready();
   ptx::pdl_wait();
   const int gid = lane >> 2;  // fragment row (column of W) / token of the B fragment
   const int t = lane & 3;     // which 32-wide k slice of the group this lane owns

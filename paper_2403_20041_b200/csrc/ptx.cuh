@@ -136,6 +136,15 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// The two halves of the cluster barrier on their own (every thread arrives once and waits once):
+// what a thread does between them does not wait for the other CTAs.
+__device__ __forceinline__ void cluster_arrive_release() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+
 // Bulk asynchronous copy global -> shared (1-D TMA); both addresses 16-byte aligned, size a
 // multiple of 16.  Completion is signalled on `bar` as transferred bytes.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes,
